@@ -1,0 +1,299 @@
+/*
+ * CAWN phase-accumulation oracle -- TEST INFRASTRUCTURE, NOT THE PRODUCT.
+ *
+ * A plain, sequential, fp64 CPU statement of what the Resonance Layer's causal
+ * phase accumulation computes.  It exists so that the CUDA library can be
+ * checked against something that can be compared with the paper by eye.  It
+ * shares no code, header, table or constant with the CUDA path and nothing in
+ * the product may call it: only the tests, the smoke check and the benchmark's
+ * CPU-baseline leg do.  Nothing here is blocked, fused, vectorised or
+ * re-associated: every function walks time once, in order.
+ *
+ * Array conventions (row-major, "complex" = two consecutive reals re, im):
+ *   pushes / outputs   [B, L, C] complex
+ *   states             [B, C]    complex
+ *   gamma, theta       [C]       (static retention and rotation per channel)
+ *   gamma_logit        [B, L, H] and freq_bias [F], C = H*F, j = h*F + k
+ *   hidden input h     [B, L, C] real;  conv weights [C, Kc];  tail [B, Kc-1, C]
+ * fp32 inputs are promoted element by element; all arithmetic is double.
+ *
+ * Pins (see tests/test_oracle_*.py): complex geometric series, prefix sum,
+ * impulse response, brute-force O(L^2) weighted sums, scipy.signal.lfilter,
+ * linearity, chunked == unchunked, gate ties, causal FIR, adjoint identity,
+ * brute-force adjoint and central finite differences.  No function in this
+ * file is "parity unpinned".
+ */
+#include <math.h>
+#include <stddef.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#define ORACLE_API __attribute__((visibility("default")))
+
+/* ------------------------------------------------------------------------ */
+/* Hard-threshold gate on Cartesian pushes (Section "Multi-Head Dynamic
+ * Parameter Projection", item Hard-Threshold Gating: a valve below epsilon is
+ * forced to exactly zero, a valve >= epsilon passes unchanged).  Read per
+ * complex channel on the phasor magnitude: open <=> |p| >= eps, decided as
+ * re^2 + im^2 >= eps^2 in double.  Both squares of fp32 values are exact in
+ * double, so the sum is rounded once whatever the compiler contracts.        */
+ORACLE_API
+void cawn_oracle_gate(int64_t n, const float *p, float gate_eps,
+                      double *z, uint8_t *mask)
+{
+    const double e2 = (double)gate_eps * (double)gate_eps;
+    for (int64_t i = 0; i < n; ++i) {
+        const double re = (double)p[2 * i], im = (double)p[2 * i + 1];
+        const int open = (re * re + im * im >= e2);
+        z[2 * i]     = open ? re : 0.0;
+        z[2 * i + 1] = open ? im : 0.0;
+        if (mask) mask[i] = (uint8_t)open;
+    }
+}
+
+/* ------------------------------------------------------------------------ */
+/* Retention of channel j = h*F + k at (b, t).
+ * Static mode: gamma[j].  Dynamic mode (Section "Multi-Head Dynamic Parameter
+ * Projection", item 4 and Frequency-Dependent Retention): a per-head logit
+ * plus a static per-harmonic bias through a sigmoid.                         */
+static double retention(const float *gamma, const float *gamma_logit,
+                        const float *freq_bias, int H, int F,
+                        int64_t bt, int j)
+{
+    if (gamma) return (double)gamma[j];
+    const int h = j / F, k = j % F;
+    const double s = (double)gamma_logit[bt * H + h] + (double)freq_bias[k];
+    return 1.0 / (1.0 + exp(-s));
+}
+
+/* ------------------------------------------------------------------------ */
+/* Causal phase accumulation, Eq. (phase_accum_r), Eq. (phase_accum_i):
+ *   P_t = z_t + gamma_t * R(theta_j) * P_{t-1},   P_{-1} = state_in (or 0)
+ * written out on real and imaginary parts exactly as the equations do.  The
+ * new push is neither decayed nor rotated; the previous state is.
+ * P_all (optional) receives the unclamped trajectory, y (optional) the output
+ * after Eq. (phase_clamp) (component-wise clamp, applied to the OUTPUT only:
+ * the recurrence and state_out carry the unclamped value).
+ * clamp_abs <= 0 disables the clamp.                                         */
+ORACLE_API
+void cawn_oracle_scan(int B, int64_t L, int H, int F,
+                      const double *z,
+                      const float *gamma, const float *theta,
+                      const float *gamma_logit, const float *freq_bias,
+                      const double *state_in, double clamp_abs,
+                      double *P_all, double *y, double *state_out)
+{
+    const int C = H * F;
+    double *Pr = (double *)malloc(sizeof(double) * (size_t)C);
+    double *Pi = (double *)malloc(sizeof(double) * (size_t)C);
+    for (int b = 0; b < B; ++b) {
+        for (int j = 0; j < C; ++j) {
+            Pr[j] = state_in ? state_in[2 * ((int64_t)b * C + j)] : 0.0;
+            Pi[j] = state_in ? state_in[2 * ((int64_t)b * C + j) + 1] : 0.0;
+        }
+        for (int64_t t = 0; t < L; ++t) {
+            const int64_t bt = (int64_t)b * L + t;
+            for (int j = 0; j < C; ++j) {
+                const double g  = retention(gamma, gamma_logit, freq_bias, H, F, bt, j);
+                const double cs = cos((double)theta[j]), sn = sin((double)theta[j]);
+                const int64_t e = 2 * (bt * C + j);
+                const double nr = z[e]     + g * (Pr[j] * cs - Pi[j] * sn);
+                const double ni = z[e + 1] + g * (Pr[j] * sn + Pi[j] * cs);
+                Pr[j] = nr;
+                Pi[j] = ni;
+                if (P_all) { P_all[e] = nr; P_all[e + 1] = ni; }
+                if (y) {
+                    double yr = nr, yi = ni;
+                    if (clamp_abs > 0.0) {
+                        yr = yr > clamp_abs ? clamp_abs : (yr < -clamp_abs ? -clamp_abs : yr);
+                        yi = yi > clamp_abs ? clamp_abs : (yi < -clamp_abs ? -clamp_abs : yi);
+                    }
+                    y[e] = yr; y[e + 1] = yi;
+                }
+            }
+        }
+        if (state_out)
+            for (int j = 0; j < C; ++j) {
+                state_out[2 * ((int64_t)b * C + j)]     = Pr[j];
+                state_out[2 * ((int64_t)b * C + j) + 1] = Pi[j];
+            }
+    }
+    free(Pr); free(Pi);
+}
+
+/* ------------------------------------------------------------------------ */
+/* Temporal Syntax Cache prelude + phasor map + gate + push.
+ *  (1) causal depthwise conv over time, left padding Kc-1 (Section "Temporal
+ *      Syntax Cache"): u_t = bias + sum_k w[c,k] * h[t-(Kc-1)+k], rows left of
+ *      t=0 come from tail_in (the carried last Kc-1 hidden rows, Section
+ *      "Throughput and Autoregressive Efficiency": the small history buffer
+ *      of the temporal conv) or are zero.  The last tap multiplies the current
+ *      token (cross-correlation, as a framework Conv1d does).
+ *  (2) optionally clamp to [-50,50] then SiLU (same section).
+ *  (3) per-channel phasor map: magnitude m = sigmoid(x), phase = pi*tanh(x)
+ *      (the benchmark's stand-in for the dense amplitude/phase projections).
+ *  (4) hard gate on the magnitude, then Eq. (gated_push_r), Eq. (gated_push_i):
+ *      z = m * (cos phase, sin phase) when open, exactly 0 when closed.
+ * VALUES are computed in double.  The gate DECISION is an integer taken from
+ * floating point, so it is taken in the arithmetic the fp32 method uses:
+ * u32 = fmaf chain in tap order k=0..Kc-1 starting from bias (or +0.0f), all
+ * in fp32 (fmaf is correctly rounded, so this is bit-reproducible anywhere);
+ * without clamp+SiLU:  open <=> u32 >= tau, tau = logit(eps) rounded to fp32
+ *                      by the caller (sigmoid is monotone, so this is
+ *                      m >= eps without evaluating the sigmoid);
+ * with clamp+SiLU:     open <=> sigmoid(x) >= eps in double.  SiLU >= -0.2785
+ *                      so m >= 0.43 always: for eps < 0.43 every gate is open.
+ * tail_out receives the last Kc-1 hidden rows seen (tail_in rows when L is
+ * shorter than Kc-1).                                                        */
+ORACLE_API
+void cawn_oracle_prelude(int B, int64_t L, int C,
+                         const float *h, const float *w, const float *bias,
+                         int Kc, int clamp_silu,
+                         const float *tail_in, float gate_eps, float gate_tau,
+                         double *z, uint8_t *mask, float *tail_out)
+{
+    const double PI = 3.14159265358979323846;
+    const int Kh = Kc - 1;
+    for (int b = 0; b < B; ++b) {
+        for (int64_t t = 0; t < L; ++t) {
+            for (int c = 0; c < C; ++c) {
+                double u = bias ? (double)bias[c] : 0.0;
+                float u32 = bias ? bias[c] : 0.0f;
+                for (int k = 0; k < Kc; ++k) {
+                    const int64_t s = t - Kh + k;      /* source time step */
+                    float hv;
+                    if (s >= 0)       hv = h[((int64_t)b * L + s) * C + c];
+                    else if (tail_in) hv = tail_in[((int64_t)b * Kh + (Kh + s)) * C + c];
+                    else              hv = 0.0f;
+                    u  += (double)w[(int64_t)c * Kc + k] * (double)hv;
+                    u32 = fmaf(w[(int64_t)c * Kc + k], hv, u32);
+                }
+                double x = u;
+                int open;
+                if (clamp_silu) {
+                    x = x > 50.0 ? 50.0 : (x < -50.0 ? -50.0 : x);
+                    x = x / (1.0 + exp(-x));
+                }
+                const double m  = 1.0 / (1.0 + exp(-x));
+                const double ph = PI * tanh(x);
+                if (clamp_silu) open = (m >= (double)gate_eps);
+                else            open = (u32 >= gate_tau);
+                const int64_t e = ((int64_t)b * L + t) * C + c;
+                z[2 * e]     = open ? m * cos(ph) : 0.0;
+                z[2 * e + 1] = open ? m * sin(ph) : 0.0;
+                if (mask) mask[e] = (uint8_t)open;
+            }
+        }
+        if (tail_out)
+            for (int r = 0; r < Kh; ++r) {
+                const int64_t s = L - Kh + r;          /* source time step */
+                for (int c = 0; c < C; ++c) {
+                    float hv;
+                    if (s >= 0)       hv = h[((int64_t)b * L + s) * C + c];
+                    else if (tail_in) hv = tail_in[((int64_t)b * Kh + (Kh + s)) * C + c];
+                    else              hv = 0.0f;
+                    tail_out[((int64_t)b * Kh + r) * C + c] = hv;
+                }
+            }
+    }
+}
+
+/* ------------------------------------------------------------------------ */
+/* Reverse-time adjoint of the accumulation (the custom backward the paper
+ * describes in Section "Complex Domain Synthesis and Hardware Compilation":
+ * gradients for the pushes and the retention; the rotation and initial-state
+ * gradients are the benchmark's additions).
+ *
+ * With the real loss  Loss = sum Re(conj(G_t) y_t) + Re(conj(dS_out) P_{L-1})
+ * and the clamp treated as pass-through (the paper: hitting the bound does not
+ * stop the gradient), the adjoint state is
+ *   lam_t = G_t + conj(a_{t+1}) lam_{t+1},  lam_{L-1} = G_{L-1} + dS_out,
+ *   a_t = gamma_t e^{i theta}.
+ * The hard gate is a straight-through estimator: d z / d p = identity, so the
+ * push gradient is lam_t at every position, open or closed.
+ *   d gamma_t(b,t,j)  = Re(conj(lam_t) e^{i theta_j} P_{t-1})
+ *   d theta_j        += Re(conj(lam_t) i a_t P_{t-1})
+ *   d state_in        = conj(a_0) lam_0
+ * Static mode sums d gamma_t over (b,t) into dgamma[C].  Dynamic mode chains
+ * through the sigmoid: s = gamma(1-gamma) d gamma_t, added to
+ * dgamma_logit[b,t,h] (sum over k) and dfreq_bias[k] (sum over b,t,h).
+ * z is the gated push trajectory (double) that the forward consumed; the
+ * forward trajectory is recomputed here, sequentially, and kept.
+ * grad_clamp_abs > 0 clamps the returned dp and dgamma component-wise (same
+ * section); <= 0 disables.                                                   */
+ORACLE_API
+void cawn_oracle_scan_bwd(int B, int64_t L, int H, int F,
+                          const double *z,
+                          const float *gamma, const float *theta,
+                          const float *gamma_logit, const float *freq_bias,
+                          const double *state_in,
+                          const float *G, const double *dstate_out,
+                          double grad_clamp_abs,
+                          double *dp, double *dgamma, double *dtheta,
+                          double *dstate_in,
+                          double *dgamma_logit, double *dfreq_bias)
+{
+    const int C = H * F;
+    const size_t n = (size_t)B * (size_t)L * (size_t)C;
+    double *P = (double *)malloc(sizeof(double) * 2 * (n ? n : 1));
+    cawn_oracle_scan(B, L, H, F, z, gamma, theta, gamma_logit, freq_bias,
+                     state_in, 0.0, P, NULL, NULL);
+
+    if (dgamma) memset(dgamma, 0, sizeof(double) * (size_t)C);
+    if (dtheta) memset(dtheta, 0, sizeof(double) * (size_t)C);
+    if (dgamma_logit) memset(dgamma_logit, 0, sizeof(double) * (size_t)B * (size_t)L * (size_t)H);
+    if (dfreq_bias) memset(dfreq_bias, 0, sizeof(double) * (size_t)F);
+
+    for (int b = 0; b < B; ++b) {
+        for (int j = 0; j < C; ++j) {
+            const double cs = cos((double)theta[j]), sn = sin((double)theta[j]);
+            /* carry = conj(a_{t+1}) lam_{t+1}; at t = L-1 it is dS_out */
+            double cr = dstate_out ? dstate_out[2 * ((int64_t)b * C + j)] : 0.0;
+            double ci = dstate_out ? dstate_out[2 * ((int64_t)b * C + j) + 1] : 0.0;
+            for (int64_t t = L - 1; t >= 0; --t) {
+                const int64_t bt = (int64_t)b * L + t;
+                const int64_t e = 2 * (bt * C + j);
+                const double lr = (double)G[e] + cr;
+                const double li = (double)G[e + 1] + ci;
+                if (dp) { dp[e] = lr; dp[e + 1] = li; }
+                /* previous state P_{t-1} */
+                double qr, qi;
+                if (t > 0) { qr = P[e - 2 * C]; qi = P[e - 2 * C + 1]; }
+                else if (state_in) { qr = state_in[2 * ((int64_t)b * C + j)];
+                                     qi = state_in[2 * ((int64_t)b * C + j) + 1]; }
+                else { qr = 0.0; qi = 0.0; }
+                const double g = retention(gamma, gamma_logit, freq_bias, H, F, bt, j);
+                /* rotated previous state  R = e^{i theta} P_{t-1} */
+                const double rr = qr * cs - qi * sn;
+                const double ri = qr * sn + qi * cs;
+                /* Re(conj(lam) R) and Re(conj(lam) i g R) = g (-lr*ri + li*rr) */
+                const double dg = lr * rr + li * ri;
+                const double dth = g * (li * rr - lr * ri);
+                if (dtheta) dtheta[j] += dth;
+                if (gamma) {
+                    if (dgamma) dgamma[j] += dg;
+                } else {
+                    const double s = g * (1.0 - g) * dg;
+                    if (dgamma_logit) dgamma_logit[bt * H + j / F] += s;
+                    if (dfreq_bias) dfreq_bias[j % F] += s;
+                }
+                /* conj(a_t) lam_t : conj(a) = g (cs - i sn) */
+                cr = g * (lr * cs + li * sn);
+                ci = g * (li * cs - lr * sn);
+            }
+            if (dstate_in) {
+                dstate_in[2 * ((int64_t)b * C + j)]     = cr;
+                dstate_in[2 * ((int64_t)b * C + j) + 1] = ci;
+            }
+        }
+    }
+    if (grad_clamp_abs > 0.0) {
+        const double c = grad_clamp_abs;
+        if (dp) for (size_t i = 0; i < 2 * n; ++i)
+            dp[i] = dp[i] > c ? c : (dp[i] < -c ? -c : dp[i]);
+        if (dgamma) for (int j = 0; j < C; ++j)
+            dgamma[j] = dgamma[j] > c ? c : (dgamma[j] < -c ? -c : dgamma[j]);
+    }
+    free(P);
+}
