@@ -1,0 +1,204 @@
+/*
+ * libcawn -- causal phase accumulation of the CAWN Resonance Layer on NVIDIA B200 (sm_100a).
+ *
+ * C ABI.  Every pointer is caller-owned; "device" pointers are CUDA global memory of the
+ * current device, "host" pointers are ordinary (preferably pinned) host memory.  The
+ * library allocates no memory and keeps no state of its own: scratch lives in a
+ * caller-provided workspace.  Calls are asynchronous on the given CUDA stream
+ * (a cudaStream_t passed as void*; NULL = the legacy default stream) unless stated.
+ *
+ * Shapes.  B batch, L time steps, H heads, F harmonics per head, C = H*F complex channels,
+ * flat channel index j = h*F + k.  "complex64" = two consecutive floats (re, im).
+ *   pushes / outputs / gradients   [B, L, C] complex64, C contiguous
+ *   states                         [B, C]    complex64
+ *   gamma, theta                   [C]       float   (retention, rotation in rad/step)
+ *   gate mask                      [B, L, ceil(C/32)] uint32, bit (j%32) of word j/32
+ * Arrays of shape [B,L,*] and the workspace must be 16-byte aligned, the others 8-byte.
+ *
+ * The operation (paper: Section "Causal Phase Accumulation and Positional Injection").
+ *   z_t   = p_t if |p_t| >= gate_eps else 0               hard-threshold gate
+ *   P_t   = z_t + gamma_j e^{i theta_j} P_{t-1}           Eq. (phase_accum_r), Eq. (phase_accum_i)
+ *   P_-1  = state_in (0 when NULL)
+ *   y_t   = clamp(P_t, +-clamp_abs) component-wise        Eq. (phase_clamp); output only
+ *   state_out = P_{L-1}, never clamped                    O(1) state passing
+ * All arithmetic is float32 on float32 data; per-channel coefficients are prepared in
+ * double inside the kernels.
+ *
+ * Errors.  Every entry point returns a cawn_status.  Negative values mean the call was
+ * rejected before anything was launched.  Conditions found on the device (a carry wait that
+ * ran out) are recorded in the workspace and read with cawn_poll_status().  Nothing aborts,
+ * traps or waits without a bound.
+ */
+#ifndef CAWN_H_
+#define CAWN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define CAWN_API __attribute__((visibility("default")))
+#else
+#define CAWN_API
+#endif
+
+typedef enum cawn_status {
+    CAWN_OK                       = 0,
+    CAWN_ERR_INVALID_ARG          = -1,  /* bad struct_size, negative size, unknown op/flag     */
+    CAWN_ERR_NULL_POINTER         = -2,  /* a required pointer is NULL                           */
+    CAWN_ERR_MISALIGNED           = -3,  /* a pointer breaks the alignment rule above            */
+    CAWN_ERR_UNSUPPORTED          = -4,  /* valid request this build has no kernel for           */
+    CAWN_ERR_WORKSPACE_TOO_SMALL  = -5,
+    CAWN_ERR_CUDA                 = -6,  /* a CUDA runtime call failed (launch, copy)            */
+    CAWN_ERR_CARRY_TIMEOUT        = 1    /* device: an inter-tile carry wait hit its bound;
+                                            outputs of that call are incomplete                  */
+} cawn_status;
+
+enum {
+    CAWN_FLAG_PRELUDE_CLAMP_SILU = 1u << 0, /* fused path: clamp conv output to +-50, then SiLU   */
+    CAWN_FLAG_RETENTION_DYNAMIC  = 1u << 1  /* gamma_t = sigmoid(gamma_logit[b,t,h] + freq_bias[k]) */
+};
+
+/* Operation selector of cawn_workspace_bytes(). */
+enum {
+    CAWN_OP_FWD        = 0,  /* workspace of cawn_phase_accumulate_fwd                           */
+    CAWN_OP_BWD_SAVED  = 1,  /* workspace of cawn_phase_accumulate_bwd with CAWN_SAVED_STATES    */
+    CAWN_OP_BWD_PUSHES = 2,  /* ... with CAWN_SAVED_PUSHES (adds room for the recomputed states) */
+    CAWN_OP_STATE      = 3,  /* size of one state blob                                           */
+    CAWN_OP_FWD_HOST   = 4   /* device staging + workspace of cawn_phase_accumulate_fwd_host     */
+};
+
+/* What the backward was given to rebuild P_{t-1} from. */
+enum {
+    CAWN_SAVED_STATES = 0,   /* the forward's unclamped outputs P [B,L,C]                        */
+    CAWN_SAVED_PUSHES = 1    /* the forward's input pushes p [B,L,C]; P is recomputed            */
+};
+
+/* Plain-data description of one call.  Fill struct_size with sizeof(cawn_params). */
+typedef struct cawn_params {
+    uint32_t struct_size;
+    int32_t  B;              /* batch >= 1                                                       */
+    int64_t  L;              /* time steps of this call, >= 0, any value (ragged is fine)        */
+    int32_t  H, F;           /* C = H*F >= 1                                                     */
+    float    gate_eps;       /* hard-gate threshold on |p| (fused path: on the magnitude m);
+                                0 = always open                                                  */
+    float    gate_tau;       /* fused path only: logit(gate_eps) rounded to float by the caller;
+                                the gate is decided as conv_output >= gate_tau                   */
+    float    clamp_abs;      /* output clamp bound (paper: 100); <= 0 disables                   */
+    float    grad_clamp_abs; /* backward: clamp returned grad_p and grad_gamma (paper: 100);
+                                <= 0 disables                                                    */
+    int32_t  conv_k;         /* fused path: conv taps 1..4; 0 = input is Cartesian pushes        */
+    uint32_t flags;          /* CAWN_FLAG_*                                                      */
+} cawn_params;
+
+/* State blob: P [B,C] complex64 (unclamped), then, at the next 16-byte boundary, the conv
+ * history [B, conv_k-1, C] float (raw hidden rows; absent when conv_k <= 1).  This is the
+ * fixed-size state the paper carries between chunks, micro-batches and decode steps
+ * (Section "Theoretical Advantages", O(1) state passing; Section "Throughput and
+ * Autoregressive Efficiency", the 2-step conv history).                                        */
+
+CAWN_API const char *cawn_status_string(int status);
+
+/* Host-only size query.  *bytes receives the size for `op` at these params. */
+CAWN_API int cawn_workspace_bytes(const cawn_params *params, int op, size_t *bytes);
+
+/* Zero a freshly allocated workspace (device).  Must run once before its first use; afterwards
+ * the kernels keep it consistent themselves.  One workspace serves one call at a time: calls
+ * that may overlap on the device need a workspace each.                                         */
+CAWN_API int cawn_workspace_init(void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * Forward phase accumulation (Eq. (gated_push_r/i) gate, Eq. (phase_accum_r/i), Eq. (phase_clamp)).
+ *
+ * conv_k == 0:  `input` = pushes p [B,L,C] complex64 (device).  y may alias input.
+ * conv_k >= 1:  fused Resonance mixing path.  `input` = hidden states h [B,L,C] float (device);
+ *               u_t = bias + sum_k conv_w[c,k] h[t-(conv_k-1)+k]   (causal depthwise conv,
+ *               Section "Temporal Syntax Cache"; rows left of t=0 from the state blob or zero),
+ *               optional clamp+-50 and SiLU, magnitude m = sigmoid(x), phase = pi*tanh(x),
+ *               gate, z = m (cos, sin)(phase).
+ * gamma/theta:  [C] device.  With CAWN_FLAG_RETENTION_DYNAMIC gamma is ignored and
+ *               gamma_logit [B,L,H], freq_bias [F] (device) define the retention
+ *               (Section "Multi-Head Dynamic Parameter Projection", item 4).
+ * state_in:     state blob (device) or NULL for a zero state.
+ * y:            [B,L,C] complex64 (device), clamped if clamp_abs > 0.
+ * state_out:    state blob (device) or NULL.  May alias state_in.
+ * gate_mask:    bit-packed mask (device) or NULL.
+ * workspace:    device, >= cawn_workspace_bytes(CAWN_OP_FWD), initialised once.
+ */
+CAWN_API int cawn_phase_accumulate_fwd(const cawn_params *params,
+                                       const void *input,
+                                       const float *gamma, const float *theta,
+                                       const float *conv_w, const float *conv_bias,
+                                       const float *gamma_logit, const float *freq_bias,
+                                       const void *state_in,
+                                       void *y, void *state_out, uint32_t *gate_mask,
+                                       void *workspace, size_t workspace_bytes,
+                                       void *cuda_stream);
+
+/*
+ * Backward of the Cartesian forward (the reverse-time adjoint the paper's custom autograd
+ * function computes, Section "Complex Domain Synthesis and Hardware Compilation").
+ *   lam_t = grad_y_t + conj(a) lam_{t+1},  lam_{L-1} = grad_y_{L-1} + grad_state_out
+ *   grad_p_t = lam_t at every position (straight-through gate; clamp passes gradient)
+ *   grad_gamma_j = sum_{b,t} Re(conj(lam_t) e^{i theta_j} P_{t-1})
+ *   grad_theta_j = sum_{b,t} Re(conj(lam_t) i a_j P_{t-1})
+ *   grad_state_in = conj(a) lam_0
+ * saved / saved_kind: CAWN_SAVED_STATES -> the forward's UNCLAMPED y; CAWN_SAVED_PUSHES -> the
+ *               forward's pushes (re-gated and re-scanned into the workspace first).
+ * grad_y:       [B,L,C] complex64 (device).  grad_p may alias it.
+ * grad_state_out, state_in: [B,C] complex64 (device) or NULL (= 0).
+ * grad_gamma, grad_theta: [C] float (device) or NULL.  grad_state_in: [B,C] complex64 or NULL.
+ * Deterministic: partial sums are combined in a fixed order in double.
+ * Static retention only.
+ */
+CAWN_API int cawn_phase_accumulate_bwd(const cawn_params *params,
+                                       const void *saved, int saved_kind,
+                                       const float *gamma, const float *theta,
+                                       const void *state_in,
+                                       const void *grad_y, const void *grad_state_out,
+                                       void *grad_p, float *grad_gamma, float *grad_theta,
+                                       void *grad_state_in,
+                                       void *workspace, size_t workspace_bytes,
+                                       void *cuda_stream);
+
+/*
+ * Associative combine of two segment summaries (static retention):
+ *   state_out = a^n_steps * state_prev + state_local,   a_j = gamma_j e^{i theta_j}
+ * where state_local is the end state of an n_steps-long segment run from a ZERO state.  This is
+ * the O(1) state passing of the paper composed outside a call (prefill that skips outputs,
+ * time sharding).  All states [B,C] complex64 (device); state_out may alias either input.
+ * a^n is evaluated in double (pow, sincos), not by repeated multiplication.
+ */
+CAWN_API int cawn_state_carry(const cawn_params *params,
+                              const void *state_prev, const void *state_local,
+                              int64_t n_steps,
+                              const float *gamma, const float *theta,
+                              void *state_out, void *cuda_stream);
+
+/* Synchronise `cuda_stream` and return the device-side status recorded in the workspace by
+ * the calls so far (CAWN_OK or a positive cawn_status); the record is then cleared.            */
+CAWN_API int cawn_poll_status(void *workspace, void *cuda_stream);
+
+/*
+ * Host-buffer convenience for the Cartesian forward: copies pushes, gamma, theta (and
+ * state_in) from HOST memory to the device staging area, runs the forward, copies y
+ * (and state_out, gate_mask) back to HOST memory, all on `cuda_stream`, and returns without
+ * synchronising.  `device_scratch` (device, >= cawn_workspace_bytes(CAWN_OP_FWD_HOST), zeroed
+ * once with cawn_workspace_init) holds staging and workspace.  Static retention, conv_k == 0.
+ */
+CAWN_API int cawn_phase_accumulate_fwd_host(const cawn_params *params,
+                                            const void *p_host,
+                                            const float *gamma_host, const float *theta_host,
+                                            const void *state_in_host,
+                                            void *y_host, void *state_out_host,
+                                            uint32_t *gate_mask_host,
+                                            void *device_scratch, size_t device_scratch_bytes,
+                                            void *cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CAWN_H_ */

@@ -87,6 +87,9 @@ void cawn_oracle_scan(int B, int64_t L, int H, int F,
     const int C = H * F;
     double *Pr = (double *)malloc(sizeof(double) * (size_t)C);
     double *Pi = (double *)malloc(sizeof(double) * (size_t)C);
+    double *cs_j = (double *)malloc(sizeof(double) * (size_t)C);   /* cos theta_j, sin theta_j */
+    double *sn_j = (double *)malloc(sizeof(double) * (size_t)C);
+    for (int j = 0; j < C; ++j) { cs_j[j] = cos((double)theta[j]); sn_j[j] = sin((double)theta[j]); }
     for (int b = 0; b < B; ++b) {
         for (int j = 0; j < C; ++j) {
             Pr[j] = state_in ? state_in[2 * ((int64_t)b * C + j)] : 0.0;
@@ -96,7 +99,7 @@ void cawn_oracle_scan(int B, int64_t L, int H, int F,
             const int64_t bt = (int64_t)b * L + t;
             for (int j = 0; j < C; ++j) {
                 const double g  = retention(gamma, gamma_logit, freq_bias, H, F, bt, j);
-                const double cs = cos((double)theta[j]), sn = sin((double)theta[j]);
+                const double cs = cs_j[j], sn = sn_j[j];
                 const int64_t e = 2 * (bt * C + j);
                 const double nr = z[e]     + g * (Pr[j] * cs - Pi[j] * sn);
                 const double ni = z[e + 1] + g * (Pr[j] * sn + Pi[j] * cs);
@@ -119,7 +122,7 @@ void cawn_oracle_scan(int B, int64_t L, int H, int F,
                 state_out[2 * ((int64_t)b * C + j) + 1] = Pi[j];
             }
     }
-    free(Pr); free(Pi);
+    free(Pr); free(Pi); free(cs_j); free(sn_j);
 }
 
 /* ------------------------------------------------------------------------ */

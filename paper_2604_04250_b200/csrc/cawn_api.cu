@@ -1,0 +1,392 @@
+// libcawn: C-ABI entry points, argument validation, workspace layout and kernel launches.
+#include "../../include/cawn.h"
+#include "cawn_scan.cuh"
+
+#include <math.h>
+#include <string.h>
+
+namespace {
+
+using namespace cawn;
+
+constexpr unsigned kPollLimit = 1u << 20;   // ~1 s of polling before a carry wait gives up
+
+inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+inline bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+// Tile shape of the scan kernels.  Long calls use 128-step tiles (8 warps x 16 steps); short
+// ones (decode, tiny chunks) use 16-step tiles so that a call is not one mostly empty CTA.
+struct TileShape { int T, W; };
+inline TileShape fwd_shape(int64_t L) { return L > 32 ? TileShape{16, 8} : TileShape{4, 4}; }
+inline TileShape bwd_shape(int64_t L) { return L > 32 ? TileShape{8, 8} : TileShape{4, 4}; }
+
+struct Geometry {
+    int C, G, K, MW;
+    size_t rec_bytes;
+};
+inline Geometry geometry(const cawn_params *p, TileShape ts)
+{
+    Geometry g;
+    g.C = p->H * p->F;
+    g.G = (g.C + 63) / 64;
+    const int64_t tile = (int64_t)ts.T * ts.W;
+    g.K = (int)((p->L + tile - 1) / tile);
+    if (g.K < 1) g.K = 1;
+    g.MW = (g.C + 31) / 32;
+    g.rec_bytes = (size_t)p->B * g.G * g.K * 64 * sizeof(uint4);
+    return g;
+}
+
+int check_params(const cawn_params *p)
+{
+    if (p == nullptr) return CAWN_ERR_NULL_POINTER;
+    if (p->struct_size != sizeof(cawn_params)) return CAWN_ERR_INVALID_ARG;
+    if (p->B < 1 || p->L < 0 || p->H < 1 || p->F < 1) return CAWN_ERR_INVALID_ARG;
+    if ((int64_t)p->H * p->F > (1 << 24)) return CAWN_ERR_INVALID_ARG;
+    if (p->conv_k < 0) return CAWN_ERR_INVALID_ARG;
+    if (p->flags & ~(uint32_t)(CAWN_FLAG_PRELUDE_CLAMP_SILU | CAWN_FLAG_RETENTION_DYNAMIC))
+        return CAWN_ERR_INVALID_ARG;
+    if (!(p->gate_eps >= 0.f)) return CAWN_ERR_INVALID_ARG;
+    return CAWN_OK;
+}
+
+size_t state_blob_bytes(const cawn_params *p)
+{
+    const size_t C = (size_t)p->H * p->F;
+    size_t n = round_up((size_t)p->B * C * sizeof(float2), 16);
+    if (p->conv_k > 1) n += round_up((size_t)p->B * (p->conv_k - 1) * C * sizeof(float), 16);
+    return n;
+}
+
+// Grid size check: tiles are a 1-D grid.
+inline bool grid_ok(const cawn_params *p, const Geometry &g)
+{
+    return (double)p->B * g.G * g.K < 2147483647.0;
+}
+
+template <int T, int W, int KIND>
+cudaError_t launch_scan(const ScanParams &sp, cudaStream_t st)
+{
+    const unsigned grid = (unsigned)((long long)sp.B * sp.G * sp.K);
+    cawn_scan_kernel<T, W, KIND><<<grid, W * 32, 0, st>>>(sp);
+    return cudaGetLastError();
+}
+
+template <int KIND>
+cudaError_t launch_scan_shape(TileShape ts, const ScanParams &sp, cudaStream_t st)
+{
+    if (ts.T == 16 && ts.W == 8) return launch_scan<16, 8, KIND>(sp, st);
+    if (ts.T == 8 && ts.W == 8) return launch_scan<8, 8, KIND>(sp, st);
+    return launch_scan<4, 4, KIND>(sp, st);
+}
+
+// Host-staged forward: layout of the device scratch.
+struct HostStage {
+    size_t off_x, off_gamma, off_theta, off_state, off_mask, off_ws, total;
+};
+HostStage host_stage(const cawn_params *p)
+{
+    const Geometry g = geometry(p, fwd_shape(p->L));
+    const size_t n = (size_t)p->B * (size_t)p->L * g.C;
+    HostStage h;
+    size_t o = 0;
+    h.off_x = o;      o += round_up(n * sizeof(float2), 256);
+    h.off_gamma = o;  o += round_up((size_t)g.C * sizeof(float), 256);
+    h.off_theta = o;  o += round_up((size_t)g.C * sizeof(float), 256);
+    h.off_state = o;  o += round_up((size_t)p->B * g.C * sizeof(float2), 256);
+    h.off_mask = o;   o += round_up((size_t)p->B * (size_t)p->L * g.MW * sizeof(uint32_t), 256);
+    h.off_ws = o;     o += sizeof(WsHeader) + g.rec_bytes;
+    h.total = o;
+    return h;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char *cawn_status_string(int status)
+{
+    switch (status) {
+    case CAWN_OK: return "ok";
+    case CAWN_ERR_INVALID_ARG: return "invalid argument";
+    case CAWN_ERR_NULL_POINTER: return "required pointer is NULL";
+    case CAWN_ERR_MISALIGNED: return "pointer is not sufficiently aligned";
+    case CAWN_ERR_UNSUPPORTED: return "request not supported by this build";
+    case CAWN_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case CAWN_ERR_CUDA: return "CUDA runtime error";
+    case CAWN_ERR_CARRY_TIMEOUT: return "device: inter-tile carry wait ran out";
+    default: return "unknown status";
+    }
+}
+
+int cawn_workspace_bytes(const cawn_params *params, int op, size_t *bytes)
+{
+    int rc = check_params(params);
+    if (rc != CAWN_OK) return rc;
+    if (bytes == nullptr) return CAWN_ERR_NULL_POINTER;
+    const size_t n = (size_t)params->B * (size_t)params->L * (size_t)params->H * params->F;
+    switch (op) {
+    case CAWN_OP_FWD: {
+        const Geometry g = geometry(params, fwd_shape(params->L));
+        *bytes = sizeof(WsHeader) + g.rec_bytes;
+        return CAWN_OK;
+    }
+    case CAWN_OP_BWD_SAVED:
+    case CAWN_OP_BWD_PUSHES: {
+        const Geometry gb = geometry(params, bwd_shape(params->L));
+        const Geometry gf = geometry(params, fwd_shape(params->L));
+        size_t rec = gb.rec_bytes > gf.rec_bytes ? gb.rec_bytes : gf.rec_bytes;
+        size_t total = sizeof(WsHeader) + round_up(rec, 256);
+        total += round_up((size_t)params->B * gb.K * gb.C * sizeof(float2), 256);
+        if (op == CAWN_OP_BWD_PUSHES) total += round_up(n * sizeof(float2), 256);
+        *bytes = total;
+        return CAWN_OK;
+    }
+    case CAWN_OP_STATE:
+        *bytes = state_blob_bytes(params);
+        return CAWN_OK;
+    case CAWN_OP_FWD_HOST:
+        *bytes = host_stage(params).total;
+        return CAWN_OK;
+    default:
+        return CAWN_ERR_INVALID_ARG;
+    }
+}
+
+int cawn_workspace_init(void *workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    if (workspace == nullptr) return CAWN_ERR_NULL_POINTER;
+    if (!aligned(workspace, 16)) return CAWN_ERR_MISALIGNED;
+    if (workspace_bytes < sizeof(WsHeader)) return CAWN_ERR_WORKSPACE_TOO_SMALL;
+    if (cudaMemsetAsync(workspace, 0, workspace_bytes, (cudaStream_t)cuda_stream) != cudaSuccess)
+        return CAWN_ERR_CUDA;
+    return CAWN_OK;
+}
+
+int cawn_phase_accumulate_fwd(const cawn_params *params, const void *input,
+                              const float *gamma, const float *theta,
+                              const float *conv_w, const float *conv_bias,
+                              const float *gamma_logit, const float *freq_bias,
+                              const void *state_in, void *y, void *state_out,
+                              uint32_t *gate_mask, void *workspace, size_t workspace_bytes,
+                              void *cuda_stream)
+{
+    int rc = check_params(params);
+    if (rc != CAWN_OK) return rc;
+    (void)conv_w; (void)conv_bias; (void)gamma_logit; (void)freq_bias;
+    if (params->conv_k != 0 || (params->flags & CAWN_FLAG_RETENTION_DYNAMIC))
+        return CAWN_ERR_UNSUPPORTED;
+    if (gamma == nullptr || theta == nullptr || workspace == nullptr) return CAWN_ERR_NULL_POINTER;
+    if (params->L > 0 && (input == nullptr || y == nullptr)) return CAWN_ERR_NULL_POINTER;
+    if (!aligned(input, 16) || !aligned(y, 16) || !aligned(workspace, 16) ||
+        !aligned(gate_mask, 4) || !aligned(state_in, 8) || !aligned(state_out, 8) ||
+        !aligned(gamma, 4) || !aligned(theta, 4))
+        return CAWN_ERR_MISALIGNED;
+    const TileShape ts = fwd_shape(params->L);
+    const Geometry g = geometry(params, ts);
+    if (!grid_ok(params, g)) return CAWN_ERR_UNSUPPORTED;
+    if (workspace_bytes < sizeof(WsHeader) + g.rec_bytes) return CAWN_ERR_WORKSPACE_TOO_SMALL;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+
+    if (params->L == 0) {               // nothing to scan: the state passes through
+        if (state_out != nullptr && state_out != state_in) {
+            const size_t nb = (size_t)params->B * g.C * sizeof(float2);
+            cudaError_t e = state_in ? cudaMemcpyAsync(state_out, state_in, nb, cudaMemcpyDeviceToDevice, st)
+                                     : cudaMemsetAsync(state_out, 0, nb, st);
+            if (e != cudaSuccess) return CAWN_ERR_CUDA;
+        }
+        return CAWN_OK;
+    }
+
+    ScanParams sp;
+    memset(&sp, 0, sizeof(sp));
+    sp.in = input; sp.out = y;
+    sp.gamma = gamma; sp.theta = theta;
+    sp.state_in = reinterpret_cast<const float2 *>(state_in);
+    sp.state_out = reinterpret_cast<float2 *>(state_out);
+    sp.mask = gate_mask;
+    sp.ws = reinterpret_cast<WsHeader *>(workspace);
+    sp.rec = reinterpret_cast<uint4 *>(reinterpret_cast<char *>(workspace) + sizeof(WsHeader));
+    sp.L = params->L; sp.B = params->B; sp.C = g.C; sp.G = g.G; sp.K = g.K; sp.MW = g.MW;
+    sp.eps2 = (double)params->gate_eps * (double)params->gate_eps;
+    sp.clampv = params->clamp_abs > 0.f ? params->clamp_abs : 0.f;
+    sp.poll_limit = kPollLimit;
+    if (launch_scan_shape<KIND_FWD>(ts, sp, st) != cudaSuccess) return CAWN_ERR_CUDA;
+    return CAWN_OK;
+}
+
+int cawn_phase_accumulate_bwd(const cawn_params *params, const void *saved, int saved_kind,
+                              const float *gamma, const float *theta, const void *state_in,
+                              const void *grad_y, const void *grad_state_out,
+                              void *grad_p, float *grad_gamma, float *grad_theta,
+                              void *grad_state_in, void *workspace, size_t workspace_bytes,
+                              void *cuda_stream)
+{
+    int rc = check_params(params);
+    if (rc != CAWN_OK) return rc;
+    if (params->conv_k != 0 || (params->flags & CAWN_FLAG_RETENTION_DYNAMIC))
+        return CAWN_ERR_UNSUPPORTED;
+    if (saved_kind != CAWN_SAVED_STATES && saved_kind != CAWN_SAVED_PUSHES) return CAWN_ERR_INVALID_ARG;
+    if (gamma == nullptr || theta == nullptr || workspace == nullptr) return CAWN_ERR_NULL_POINTER;
+    const bool want_param = (grad_gamma != nullptr || grad_theta != nullptr);
+    if (params->L > 0 && (grad_y == nullptr || grad_p == nullptr)) return CAWN_ERR_NULL_POINTER;
+    if (params->L > 0 && want_param && saved == nullptr) return CAWN_ERR_NULL_POINTER;
+    if (!aligned(saved, 16) || !aligned(grad_y, 16) || !aligned(grad_p, 16) || !aligned(workspace, 16) ||
+        !aligned(state_in, 8) || !aligned(grad_state_out, 8) || !aligned(grad_state_in, 8))
+        return CAWN_ERR_MISALIGNED;
+    size_t need = 0;
+    rc = cawn_workspace_bytes(params, saved_kind == CAWN_SAVED_PUSHES ? CAWN_OP_BWD_PUSHES : CAWN_OP_BWD_SAVED, &need);
+    if (rc != CAWN_OK) return rc;
+    if (workspace_bytes < need) return CAWN_ERR_WORKSPACE_TOO_SMALL;
+    const TileShape tb = bwd_shape(params->L), tf = fwd_shape(params->L);
+    const Geometry gb = geometry(params, tb), gf = geometry(params, tf);
+    if (!grid_ok(params, gb) || !grid_ok(params, gf)) return CAWN_ERR_UNSUPPORTED;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    const int C = gb.C;
+
+    if (params->L == 0) {
+        const size_t nb = (size_t)params->B * C * sizeof(float2);
+        if (grad_state_in != nullptr && grad_state_in != grad_state_out) {
+            cudaError_t e = grad_state_out ? cudaMemcpyAsync(grad_state_in, grad_state_out, nb, cudaMemcpyDeviceToDevice, st)
+                                           : cudaMemsetAsync(grad_state_in, 0, nb, st);
+            if (e != cudaSuccess) return CAWN_ERR_CUDA;
+        }
+        if (grad_gamma && cudaMemsetAsync(grad_gamma, 0, C * sizeof(float), st) != cudaSuccess) return CAWN_ERR_CUDA;
+        if (grad_theta && cudaMemsetAsync(grad_theta, 0, C * sizeof(float), st) != cudaSuccess) return CAWN_ERR_CUDA;
+        return CAWN_OK;
+    }
+
+    char *base = reinterpret_cast<char *>(workspace);
+    const size_t rec = gb.rec_bytes > gf.rec_bytes ? gb.rec_bytes : gf.rec_bytes;
+    size_t off = sizeof(WsHeader);
+    uint4 *recs = reinterpret_cast<uint4 *>(base + off);            off += round_up(rec, 256);
+    float2 *qpart = reinterpret_cast<float2 *>(base + off);         off += round_up((size_t)params->B * gb.K * C * sizeof(float2), 256);
+    float2 *Pbuf = reinterpret_cast<float2 *>(base + off);
+
+    const void *states = saved;
+    if (want_param && saved_kind == CAWN_SAVED_PUSHES) {
+        // rebuild the unclamped forward states from the pushes (gate, then scan)
+        ScanParams fp;
+        memset(&fp, 0, sizeof(fp));
+        fp.in = saved; fp.out = Pbuf;
+        fp.gamma = gamma; fp.theta = theta;
+        fp.state_in = reinterpret_cast<const float2 *>(state_in);
+        fp.ws = reinterpret_cast<WsHeader *>(workspace);
+        fp.rec = recs;
+        fp.L = params->L; fp.B = params->B; fp.C = C; fp.G = gf.G; fp.K = gf.K; fp.MW = gf.MW;
+        fp.eps2 = (double)params->gate_eps * (double)params->gate_eps;
+        fp.clampv = 0.f;
+        fp.poll_limit = kPollLimit;
+        if (launch_scan_shape<KIND_FWD>(tf, fp, st) != cudaSuccess) return CAWN_ERR_CUDA;
+        states = Pbuf;
+    }
+
+    ScanParams sp;
+    memset(&sp, 0, sizeof(sp));
+    sp.in = grad_y; sp.out = grad_p;
+    sp.aux = want_param ? states : nullptr;
+    sp.gamma = gamma; sp.theta = theta;
+    sp.state_in = reinterpret_cast<const float2 *>(state_in);
+    sp.edge_in = reinterpret_cast<const float2 *>(grad_state_out);
+    sp.state_out = reinterpret_cast<float2 *>(grad_state_in);
+    sp.ws = reinterpret_cast<WsHeader *>(workspace);
+    sp.rec = recs;
+    sp.qpart = want_param ? qpart : nullptr;
+    sp.L = params->L; sp.B = params->B; sp.C = C; sp.G = gb.G; sp.K = gb.K; sp.MW = gb.MW;
+    sp.clampv = params->grad_clamp_abs > 0.f ? params->grad_clamp_abs : 0.f;
+    sp.poll_limit = kPollLimit;
+    if (launch_scan_shape<KIND_BWD>(tb, sp, st) != cudaSuccess) return CAWN_ERR_CUDA;
+
+    if (want_param) {
+        const int warps = 8;
+        cawn_bwd_finalize_kernel<<<(C + warps - 1) / warps, warps * 32, 0, st>>>(
+            qpart, params->B * gb.K, C, gamma, theta, grad_gamma, grad_theta, sp.clampv);
+        if (cudaGetLastError() != cudaSuccess) return CAWN_ERR_CUDA;
+    }
+    return CAWN_OK;
+}
+
+int cawn_state_carry(const cawn_params *params, const void *state_prev, const void *state_local,
+                     int64_t n_steps, const float *gamma, const float *theta,
+                     void *state_out, void *cuda_stream)
+{
+    int rc = check_params(params);
+    if (rc != CAWN_OK) return rc;
+    if (n_steps < 0) return CAWN_ERR_INVALID_ARG;
+    if (params->flags & CAWN_FLAG_RETENTION_DYNAMIC) return CAWN_ERR_UNSUPPORTED;
+    if (!state_prev || !state_local || !gamma || !theta || !state_out) return CAWN_ERR_NULL_POINTER;
+    if (!aligned(state_prev, 8) || !aligned(state_local, 8) || !aligned(state_out, 8))
+        return CAWN_ERR_MISALIGNED;
+    const int C = params->H * params->F;
+    const long long n = (long long)params->B * C;
+    cawn_state_carry_kernel<<<(unsigned)((n + 255) / 256), 256, 0, (cudaStream_t)cuda_stream>>>(
+        reinterpret_cast<const float2 *>(state_prev), reinterpret_cast<const float2 *>(state_local),
+        reinterpret_cast<float2 *>(state_out), gamma, theta, n_steps, params->B, C);
+    return cudaGetLastError() == cudaSuccess ? CAWN_OK : CAWN_ERR_CUDA;
+}
+
+int cawn_poll_status(void *workspace, void *cuda_stream)
+{
+    if (workspace == nullptr) return CAWN_ERR_NULL_POINTER;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    WsHeader *ws = reinterpret_cast<WsHeader *>(workspace);
+    unsigned status = 0;
+    if (cudaMemcpyAsync(&status, &ws->status, sizeof(status), cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return CAWN_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return CAWN_ERR_CUDA;
+    if (status != 0) {
+        if (cudaMemsetAsync(&ws->status, 0, sizeof(status), st) != cudaSuccess) return CAWN_ERR_CUDA;
+        if (cudaStreamSynchronize(st) != cudaSuccess) return CAWN_ERR_CUDA;
+    }
+    return (int)status;
+}
+
+int cawn_phase_accumulate_fwd_host(const cawn_params *params, const void *p_host,
+                                   const float *gamma_host, const float *theta_host,
+                                   const void *state_in_host, void *y_host, void *state_out_host,
+                                   uint32_t *gate_mask_host, void *device_scratch,
+                                   size_t device_scratch_bytes, void *cuda_stream)
+{
+    int rc = check_params(params);
+    if (rc != CAWN_OK) return rc;
+    if (params->conv_k != 0 || (params->flags & CAWN_FLAG_RETENTION_DYNAMIC))
+        return CAWN_ERR_UNSUPPORTED;
+    if (!gamma_host || !theta_host || !device_scratch) return CAWN_ERR_NULL_POINTER;
+    if (params->L > 0 && (!p_host || !y_host)) return CAWN_ERR_NULL_POINTER;
+    if (!aligned(device_scratch, 256)) return CAWN_ERR_MISALIGNED;
+    const HostStage h = host_stage(params);
+    if (device_scratch_bytes < h.total) return CAWN_ERR_WORKSPACE_TOO_SMALL;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    char *d = reinterpret_cast<char *>(device_scratch);
+    const size_t C = (size_t)params->H * params->F;
+    const size_t n = (size_t)params->B * (size_t)params->L * C;
+    const size_t state_bytes = (size_t)params->B * C * sizeof(float2);
+    const size_t mask_bytes = (size_t)params->B * (size_t)params->L * ((C + 31) / 32) * sizeof(uint32_t);
+    bool ok = true;
+    ok &= cudaMemcpyAsync(d + h.off_gamma, gamma_host, C * sizeof(float), cudaMemcpyHostToDevice, st) == cudaSuccess;
+    ok &= cudaMemcpyAsync(d + h.off_theta, theta_host, C * sizeof(float), cudaMemcpyHostToDevice, st) == cudaSuccess;
+    if (state_in_host)
+        ok &= cudaMemcpyAsync(d + h.off_state, state_in_host, state_bytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    if (n)
+        ok &= cudaMemcpyAsync(d + h.off_x, p_host, n * sizeof(float2), cudaMemcpyHostToDevice, st) == cudaSuccess;
+    if (!ok) return CAWN_ERR_CUDA;
+    rc = cawn_phase_accumulate_fwd(params, d + h.off_x,
+                                   reinterpret_cast<const float *>(d + h.off_gamma),
+                                   reinterpret_cast<const float *>(d + h.off_theta),
+                                   nullptr, nullptr, nullptr, nullptr,
+                                   state_in_host ? d + h.off_state : nullptr,
+                                   d + h.off_x,                               /* in place */
+                                   state_out_host ? d + h.off_state : nullptr,
+                                   gate_mask_host ? reinterpret_cast<uint32_t *>(d + h.off_mask) : nullptr,
+                                   d + h.off_ws, h.total - h.off_ws, st);
+    if (rc != CAWN_OK) return rc;
+    if (n)
+        ok &= cudaMemcpyAsync(y_host, d + h.off_x, n * sizeof(float2), cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    if (state_out_host)
+        ok &= cudaMemcpyAsync(state_out_host, d + h.off_state, state_bytes, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    if (gate_mask_host && mask_bytes)
+        ok &= cudaMemcpyAsync(gate_mask_host, d + h.off_mask, mask_bytes, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    return ok ? CAWN_OK : CAWN_ERR_CUDA;
+}
+
+}  // extern "C"
