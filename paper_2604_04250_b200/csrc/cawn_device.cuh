@@ -102,8 +102,8 @@ __device__ __forceinline__ bool carry_lookback(const uint4 *chain, int k, int la
         bool progressed = false;
         if (!d0) {
             const unsigned long long tag = ((unsigned long long)r0.w << 32) | r0.z;
-            if ((tag >> 2) == epoch) {
-                const unsigned kind = (unsigned)(tag & 3ull);
+            const unsigned kind = (unsigned)(tag & 3ull);
+            if ((tag >> 2) == epoch && kind != 0u) {       // kind 0: never written (zeroed workspace)
                 progressed = true;
                 if (kind == REC_POISON || (kind != REC_PREFIX && i0 == 0)) { ok = false; d0 = true; }
                 else {
@@ -115,8 +115,8 @@ __device__ __forceinline__ bool carry_lookback(const uint4 *chain, int k, int la
         }
         if (!d1) {
             const unsigned long long tag = ((unsigned long long)r1.w << 32) | r1.z;
-            if ((tag >> 2) == epoch) {
-                const unsigned kind = (unsigned)(tag & 3ull);
+            const unsigned kind = (unsigned)(tag & 3ull);
+            if ((tag >> 2) == epoch && kind != 0u) {
                 progressed = true;
                 if (kind == REC_POISON || (kind != REC_PREFIX && i1 == 0)) { ok = false; d1 = true; }
                 else {
