@@ -20,9 +20,11 @@ struct TileShape { int T, W; };
 inline TileShape fwd_shape(int64_t L) { return L > 32 ? TileShape{16, 8} : TileShape{4, 4}; }
 inline TileShape bwd_shape(int64_t L) { return L > 32 ? TileShape{8, 8} : TileShape{4, 4}; }
 
+// C channels in G groups of 64; K tiles along time, of which every (W-1)-th is a checkpoint
+// (KP checkpoint slots per chain); MW mask words per row.  Records are 16 bytes per channel.
 struct Geometry {
-    int C, G, K, MW;
-    size_t rec_bytes;
+    int C, G, K, KP, MW;
+    size_t agg_bytes, pre_bytes, rec_bytes;
 };
 inline Geometry geometry(const cawn_params *p, TileShape ts)
 {
@@ -32,9 +34,37 @@ inline Geometry geometry(const cawn_params *p, TileShape ts)
     const int64_t tile = (int64_t)ts.T * ts.W;
     g.K = (int)((p->L + tile - 1) / tile);
     if (g.K < 1) g.K = 1;
+    g.KP = g.K / (ts.W - 1) + 1;
     g.MW = (g.C + 31) / 32;
-    g.rec_bytes = (size_t)p->B * g.G * g.K * 64 * sizeof(uint4);
+    g.agg_bytes = (size_t)p->B * g.G * g.K * 64 * sizeof(uint4);
+    g.pre_bytes = (size_t)p->B * g.G * g.KP * 64 * sizeof(uint4);
+    g.rec_bytes = g.agg_bytes + g.pre_bytes;
     return g;
+}
+
+// Carry-record area of a workspace: aggregates, then checkpoint carry-ins.
+inline void set_records(ScanParams &sp, char *rec_base, const Geometry &g)
+{
+    sp.agg = reinterpret_cast<uint4 *>(rec_base);
+    sp.pre = reinterpret_cast<uint4 *>(rec_base + g.agg_bytes);
+    sp.G = g.G; sp.K = g.K; sp.KP = g.KP; sp.MW = g.MW; sp.C = g.C;
+}
+
+// fp32 screen of the gate: the fp32 sum of squares is within 2^-22 (relative) of the exact
+// one, so outside a 2^-21 band around eps^2 it already decides the double comparison.
+inline void set_gate(ScanParams &sp, float gate_eps)
+{
+    const double e2 = (double)gate_eps * (double)gate_eps;
+    sp.eps2 = e2;
+    if (e2 == 0.0) {                       // always open (NaN inputs still compare false)
+        sp.gate_lo = 0.f; sp.gate_hi = 0.f;
+    } else if (e2 < 1e-27) {               // fp32 products may be subnormal: screen only far above
+        sp.gate_lo = 0.f; sp.gate_hi = 1e-24f;
+    } else {
+        const double band = 1.0 / 2097152.0;
+        sp.gate_lo = nextafterf((float)(e2 * (1.0 - band)), -INFINITY);
+        sp.gate_hi = nextafterf((float)(e2 * (1.0 + band)), INFINITY);
+    }
 }
 
 int check_params(const cawn_params *p)
@@ -64,11 +94,14 @@ inline bool grid_ok(const cawn_params *p, const Geometry &g)
     return (double)p->B * g.G * g.K < 2147483647.0;
 }
 
+// The float4 path needs every row segment on a 16-byte boundary: C even (the arrays
+// themselves are checked to be 16-byte aligned).
 template <int T, int W, int KIND>
 cudaError_t launch_scan(const ScanParams &sp, cudaStream_t st)
 {
     const unsigned grid = (unsigned)((long long)sp.B * sp.G * sp.K);
-    cawn_scan_kernel<T, W, KIND><<<grid, W * 32, 0, st>>>(sp);
+    if (sp.C % 2 == 0) cawn_scan_kernel<T, W, KIND, true><<<grid, W * 32, 0, st>>>(sp);
+    else               cawn_scan_kernel<T, W, KIND, false><<<grid, W * 32, 0, st>>>(sp);
     return cudaGetLastError();
 }
 
@@ -206,9 +239,9 @@ int cawn_phase_accumulate_fwd(const cawn_params *params, const void *input,
     sp.state_out = reinterpret_cast<float2 *>(state_out);
     sp.mask = gate_mask;
     sp.ws = reinterpret_cast<WsHeader *>(workspace);
-    sp.rec = reinterpret_cast<uint4 *>(reinterpret_cast<char *>(workspace) + sizeof(WsHeader));
-    sp.L = params->L; sp.B = params->B; sp.C = g.C; sp.G = g.G; sp.K = g.K; sp.MW = g.MW;
-    sp.eps2 = (double)params->gate_eps * (double)params->gate_eps;
+    set_records(sp, reinterpret_cast<char *>(workspace) + sizeof(WsHeader), g);
+    sp.L = params->L; sp.B = params->B;
+    set_gate(sp, params->gate_eps);
     sp.clampv = params->clamp_abs > 0.f ? params->clamp_abs : 0.f;
     sp.poll_limit = kPollLimit;
     if (launch_scan_shape<KIND_FWD>(ts, sp, st) != cudaSuccess) return CAWN_ERR_CUDA;
@@ -259,7 +292,7 @@ int cawn_phase_accumulate_bwd(const cawn_params *params, const void *saved, int 
     char *base = reinterpret_cast<char *>(workspace);
     const size_t rec = gb.rec_bytes > gf.rec_bytes ? gb.rec_bytes : gf.rec_bytes;
     size_t off = sizeof(WsHeader);
-    uint4 *recs = reinterpret_cast<uint4 *>(base + off);            off += round_up(rec, 256);
+    char *recs = base + off;                                        off += round_up(rec, 256);
     float2 *qpart = reinterpret_cast<float2 *>(base + off);         off += round_up((size_t)params->B * gb.K * C * sizeof(float2), 256);
     float2 *Pbuf = reinterpret_cast<float2 *>(base + off);
 
@@ -272,9 +305,9 @@ int cawn_phase_accumulate_bwd(const cawn_params *params, const void *saved, int 
         fp.gamma = gamma; fp.theta = theta;
         fp.state_in = reinterpret_cast<const float2 *>(state_in);
         fp.ws = reinterpret_cast<WsHeader *>(workspace);
-        fp.rec = recs;
-        fp.L = params->L; fp.B = params->B; fp.C = C; fp.G = gf.G; fp.K = gf.K; fp.MW = gf.MW;
-        fp.eps2 = (double)params->gate_eps * (double)params->gate_eps;
+        set_records(fp, recs, gf);
+        fp.L = params->L; fp.B = params->B;
+        set_gate(fp, params->gate_eps);
         fp.clampv = 0.f;
         fp.poll_limit = kPollLimit;
         if (launch_scan_shape<KIND_FWD>(tf, fp, st) != cudaSuccess) return CAWN_ERR_CUDA;
@@ -290,9 +323,9 @@ int cawn_phase_accumulate_bwd(const cawn_params *params, const void *saved, int 
     sp.edge_in = reinterpret_cast<const float2 *>(grad_state_out);
     sp.state_out = reinterpret_cast<float2 *>(grad_state_in);
     sp.ws = reinterpret_cast<WsHeader *>(workspace);
-    sp.rec = recs;
+    set_records(sp, recs, gb);
     sp.qpart = want_param ? qpart : nullptr;
-    sp.L = params->L; sp.B = params->B; sp.C = C; sp.G = gb.G; sp.K = gb.K; sp.MW = gb.MW;
+    sp.L = params->L; sp.B = params->B;
     sp.clampv = params->grad_clamp_abs > 0.f ? params->grad_clamp_abs : 0.f;
     sp.poll_limit = kPollLimit;
     if (launch_scan_shape<KIND_BWD>(tb, sp, st) != cudaSuccess) return CAWN_ERR_CUDA;

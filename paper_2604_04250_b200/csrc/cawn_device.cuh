@@ -1,4 +1,4 @@
-// Device-side helpers shared by the libcawn kernels: complex float arithmetic, the
+// Device-side helpers shared by the libcawn kernels: paired complex float arithmetic, the
 // workspace header, and the 16-byte tagged records the inter-tile carry protocol uses.
 #pragma once
 #include <cuda_runtime.h>
@@ -7,11 +7,12 @@
 namespace cawn {
 
 // ---------------------------------------------------------------------------------------
-// Workspace layout: [WsHeader (256 B)] [carry records] [op-specific areas]
-// epoch  : generation number of the current launch; records tagged with another epoch are
-//          stale, so nothing ever needs clearing between launches.  The last CTA of a launch
-//          bumps it.
-// done   : CTAs of the current launch that have finished (reset by the last one).
+// Workspace layout: [WsHeader (256 B)] [aggregate records] [prefix records] [op-specific areas]
+// epoch  : generation number of the current launch.  Records carry the epoch they were
+//          written in; a record of another epoch is stale, so nothing is cleared between
+//          launches (and a launch replayed from a CUDA graph still sees a fresh epoch).
+// done   : CTAs of the current launch that have read the epoch.  The last one to arrive
+//          resets the count and opens the next epoch; by then nobody reads `epoch` any more.
 // status : sticky device-side error (cawn_status > 0), cleared by cawn_poll_status.
 struct __align__(16) WsHeader {
     unsigned long long epoch;
@@ -24,19 +25,36 @@ static_assert(sizeof(WsHeader) == 256, "workspace header is 256 bytes");
 enum : unsigned { REC_AGGREGATE = 1u, REC_PREFIX = 2u, REC_POISON = 3u };
 
 // ---------------------------------------------------------------------------------------
+// Every lane works on two adjacent channels at once; a float4 holds (re0, im0, re1, im1).
 __device__ __forceinline__ float2 cmul(float2 a, float2 b)
 {
     return make_float2(fmaf(a.x, b.x, -a.y * b.y), fmaf(a.x, b.y, a.y * b.x));
 }
-// a * b + c
-__device__ __forceinline__ float2 cfma(float2 a, float2 b, float2 c)
+// a * b + c on both channels of a pair
+__device__ __forceinline__ float4 cfma2(float4 a, float4 b, float4 c)
 {
-    float2 r;
+    float4 r;
     r.x = fmaf(a.x, b.x, fmaf(-a.y, b.y, c.x));
     r.y = fmaf(a.x, b.y, fmaf(a.y, b.x, c.y));
+    r.z = fmaf(a.z, b.z, fmaf(-a.w, b.w, c.z));
+    r.w = fmaf(a.z, b.w, fmaf(a.w, b.z, c.w));
+    return r;
+}
+__device__ __forceinline__ float4 cmul2(float4 a, float4 b)
+{
+    float4 r;
+    r.x = fmaf(a.x, b.x, -a.y * b.y);
+    r.y = fmaf(a.x, b.y, a.y * b.x);
+    r.z = fmaf(a.z, b.z, -a.w * b.w);
+    r.w = fmaf(a.z, b.w, a.w * b.z);
     return r;
 }
 __device__ __forceinline__ float clampf(float v, float c) { return fminf(fmaxf(v, -c), c); }
+__device__ __forceinline__ float4 clamp4(float4 v, float c)
+{
+    return make_float4(clampf(v.x, c), clampf(v.y, c), clampf(v.z, c), clampf(v.w, c));
+}
+__device__ __forceinline__ float4 zero4() { return make_float4(0.f, 0.f, 0.f, 0.f); }
 
 // Integer power of a complex double by square-and-multiply (N is a compile-time constant).
 template <int N>
@@ -53,19 +71,19 @@ __device__ __forceinline__ void cpow_int(double ar, double ai, double &rr, doubl
 
 // ---------------------------------------------------------------------------------------
 // Carry records: {re, im, tag} in one aligned 16-byte word, written and read with single
-// 128-bit accesses so value and tag are always seen together.
-// tag = epoch * 4 + kind.
-__device__ __forceinline__ void st_record(uint4 *p, float2 v, unsigned long long tag)
+// 128-bit accesses at GPU scope so value and tag are always seen together.
+// tag = epoch * 4 + kind; kind 0 never occurs in a written record.
+__device__ __forceinline__ void st_record(uint4 *p, float re, float im, unsigned long long tag)
 {
-    asm volatile("st.volatile.global.v4.u32 [%0], {%1, %2, %3, %4};"
-                 :: "l"(p), "r"(__float_as_uint(v.x)), "r"(__float_as_uint(v.y)),
+    asm volatile("st.relaxed.gpu.global.v4.u32 [%0], {%1, %2, %3, %4};"
+                 :: "l"(p), "r"(__float_as_uint(re)), "r"(__float_as_uint(im)),
                     "r"((unsigned)(tag & 0xffffffffull)), "r"((unsigned)(tag >> 32))
                  : "memory");
 }
 __device__ __forceinline__ uint4 ld_record(const uint4 *p)
 {
     uint4 v;
-    asm volatile("ld.volatile.global.v4.u32 {%0, %1, %2, %3}, [%4];"
+    asm volatile("ld.relaxed.gpu.global.v4.u32 {%0, %1, %2, %3}, [%4];"
                  : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
     return v;
 }
@@ -79,59 +97,46 @@ __device__ __forceinline__ void st_volatile_u64(unsigned long long *p, unsigned 
 {
     asm volatile("st.volatile.global.u64 [%0], %1;" :: "l"(p), "l"(v) : "memory");
 }
-
-// One lane's look-back over the tiles before tile k of its chain, for its two channels.
-// Tile 0 of a chain always publishes a PREFIX, so the walk ends there at the latest.
-// `chain` points at the records of tile 0 (64 per tile: lane and lane+32).
-// Returns false when a wait ran out of polls or a predecessor published POISON.
-__device__ __forceinline__ bool carry_lookback(const uint4 *chain, int k, int lane,
-                                               bool v0, bool v1, unsigned long long epoch,
-                                               float2 aW0, float2 aW1, unsigned poll_limit,
-                                               float2 &S0, float2 &S1)
+__device__ __forceinline__ void st_volatile_u32(unsigned *p, unsigned v)
 {
-    int i0 = k - 1, i1 = k - 1;
-    bool d0 = !v0, d1 = !v1, ok = true;
-    float2 w0 = make_float2(1.f, 0.f), w1 = w0;
-    S0 = make_float2(0.f, 0.f);
-    S1 = S0;
+    asm volatile("st.volatile.global.u32 [%0], %1;" :: "l"(p), "r"(v) : "memory");
+}
+
+// 0 = not written in this epoch yet, else the record's kind.
+__device__ __forceinline__ unsigned record_kind(uint4 r, unsigned long long epoch)
+{
+    const unsigned long long tag = ((unsigned long long)r.w << 32) | r.z;
+    return (tag >> 2) == epoch ? (unsigned)(tag & 3ull) : 0u;
+}
+
+// Publish the two records of this lane's channel pair (lane l owns records 2l and 2l+1 of the
+// 64 that belong to one tile).
+__device__ __forceinline__ void publish_pair(uint4 *tile_recs, int lane, float4 v,
+                                             unsigned long long epoch, unsigned kind)
+{
+    const unsigned long long tag = epoch * 4ull + kind;
+    st_record(tile_recs + 2 * lane, v.x, v.y, tag);
+    st_record(tile_recs + 2 * lane + 1, v.z, v.w, tag);
+}
+
+// Wait (with a bound) until both records of this lane's pair carry `epoch`.  Returns false when
+// the wait ran out or the writer published POISON.
+__device__ __forceinline__ bool poll_pair(const uint4 *tile_recs, int lane, unsigned long long epoch,
+                                          unsigned poll_limit, float4 &v)
+{
+    const uint4 *p = tile_recs + 2 * lane;
     unsigned polls = 0;
-    while (!(d0 && d1)) {
-        uint4 r0 = make_uint4(0, 0, 0, 0), r1 = r0;
-        if (!d0) r0 = ld_record(chain + (long long)i0 * 64 + lane);
-        if (!d1) r1 = ld_record(chain + (long long)i1 * 64 + lane + 32);
-        bool progressed = false;
-        if (!d0) {
-            const unsigned long long tag = ((unsigned long long)r0.w << 32) | r0.z;
-            const unsigned kind = (unsigned)(tag & 3ull);
-            if ((tag >> 2) == epoch && kind != 0u) {       // kind 0: never written (zeroed workspace)
-                progressed = true;
-                if (kind == REC_POISON || (kind != REC_PREFIX && i0 == 0)) { ok = false; d0 = true; }
-                else {
-                    S0 = cfma(w0, make_float2(__uint_as_float(r0.x), __uint_as_float(r0.y)), S0);
-                    if (kind == REC_PREFIX) d0 = true;
-                    else { w0 = cmul(w0, aW0); --i0; }
-                }
-            }
+    for (;;) {
+        const uint4 r0 = ld_record(p), r1 = ld_record(p + 1);
+        const unsigned k0 = record_kind(r0, epoch), k1 = record_kind(r1, epoch);
+        if (k0 != 0u && k1 != 0u) {
+            v = make_float4(__uint_as_float(r0.x), __uint_as_float(r0.y),
+                            __uint_as_float(r1.x), __uint_as_float(r1.y));
+            return k0 != REC_POISON && k1 != REC_POISON;
         }
-        if (!d1) {
-            const unsigned long long tag = ((unsigned long long)r1.w << 32) | r1.z;
-            const unsigned kind = (unsigned)(tag & 3ull);
-            if ((tag >> 2) == epoch && kind != 0u) {
-                progressed = true;
-                if (kind == REC_POISON || (kind != REC_PREFIX && i1 == 0)) { ok = false; d1 = true; }
-                else {
-                    S1 = cfma(w1, make_float2(__uint_as_float(r1.x), __uint_as_float(r1.y)), S1);
-                    if (kind == REC_PREFIX) d1 = true;
-                    else { w1 = cmul(w1, aW1); --i1; }
-                }
-            }
-        }
-        if (!progressed) {
-            if (++polls > poll_limit) { ok = false; break; }
-            if (polls > 8) __nanosleep(polls > 64 ? 200 : 40);
-        }
+        if (++polls > poll_limit) { v = zero4(); return false; }
+        if (polls > 4) __nanosleep(polls > 64 ? 256 : 32);
     }
-    return ok;
 }
 
 }  // namespace cawn

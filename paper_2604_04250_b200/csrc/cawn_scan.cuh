@@ -1,22 +1,31 @@
 // The chunk-parallel phase-accumulation kernel.
 //
 // One CTA owns a tile of TILE = W*T consecutive time steps of one (batch, 64-channel group).
-// Warp w owns T consecutive steps, lane l owns channels (64g + l) and (64g + 32 + l), so every
-// warp-wide access is a run of 256 contiguous bytes and a tile row is 512 contiguous bytes.
+// Warp w owns T consecutive steps; lane l owns the adjacent channels 64g + 2l and 64g + 2l + 1,
+// so a warp-wide access is one 512-byte row segment read or written as 32 float4.
 // The tile lives in registers between its single read and its single write:
 //
-//   0. every thread issues all of its loads (T rows x 2 channels, independent);
-//      meanwhile 64 threads prepare the per-channel coefficients a, a^T, a^TILE in double
-//   1. gate (Cartesian forward), then the thread reduces its T steps from a zero start
-//   2. warp 0 folds the W partial ends into the tile aggregate, publishes it, looks back
-//      along time for the tile's carry-in (decoupled look-back over 16-byte tagged records),
-//      publishes the inclusive prefix
-//   3. every thread folds the earlier warps' ends onto the carry-in, re-runs its T steps as
-//      the plain recurrence from that state and stores the results
+//   0. every thread issues all of its loads (T rows, independent); meanwhile 64 threads
+//      prepare the per-channel coefficients a, a^T, a^TILE in double            [barrier 1]
+//   1. gate (Cartesian forward), then each thread reduces its T steps from a zero start and
+//      leaves the end state in shared memory                                     [barrier 2]
+//   2. warp 0 folds the W ends into the tile aggregate and publishes it; then every warp
+//      fetches one record of the carry window (below) into shared memory         [barrier 3]
+//   3. every warp folds the window into the tile's carry-in, folds the earlier warps' ends on
+//      top, re-runs its T steps as the plain recurrence from that state and stores them
 //
-// So each run of the fp32 recurrence is at most T steps long and everything that crosses a
-// thread boundary is multiplied by a power of a_j rounded once from double: the systematic
-// rounding error of a_j does not build up with sequence length.
+// Carry window.  With M = W-1, the tiles k = M, 2M, ... of a chain are checkpoints: they also
+// publish their carry-in X_k (the state before the tile).  Tile k reads the carry-in of the
+// last checkpoint c < k (c = 0: the call's initial state) and the aggregates E_c .. E_{k-1},
+// and evaluates X_k = A^(k-c) X_c + sum A^(k-1-i) E_i by Horner's rule, oldest first, A = a^TILE.
+// What is read and the order it is combined in depend on k alone, never on timing, so results
+// are bit-for-bit repeatable; aggregates are published before anything is waited for, so the
+// only serial dependency runs from checkpoint to checkpoint.  A tile only ever waits for tiles
+// with a smaller block index, which the hardware has dispatched before it.
+//
+// Each run of the fp32 recurrence is at most T steps long and everything that crosses a thread
+// boundary is multiplied by a power of a_j rounded once from double: the rounding error of
+// a_j does not build up with sequence length.
 //
 // The backward is the same operator run right-to-left with conj(a_j); it additionally
 // accumulates sum conj(lam_t) P_{t-1} per channel for the retention and rotation gradients.
@@ -37,84 +46,99 @@ struct ScanParams {
     float2 *state_out;           // FWD: state_out;  BWD: grad_state_in
     uint32_t *mask;              // FWD: bit-packed gate mask or NULL
     WsHeader *ws;
-    uint4 *rec;                  // carry records [B][G][K][64]
+    uint4 *agg;                  // aggregate records [B][G][K][64]
+    uint4 *pre;                  // checkpoint carry-in records [B][G][KP][64]
     float2 *qpart;               // BWD: per-tile partial sums [B*K][C]
     long long L;
-    int B, C, G, K, MW;          // MW = mask words per row
+    int B, C, G, K, KP, MW;      // MW = mask words per row
     double eps2;                 // gate threshold squared
+    float gate_lo, gate_hi;      // fp32 screen: below lo surely closed, at or above hi surely open
     float clampv;                // output (FWD) or gradient (BWD) clamp; <= 0 off
     unsigned poll_limit;
 };
 
-template <int T, int W, int KIND>
-__global__ void __launch_bounds__(W * 32) cawn_scan_kernel(const ScanParams prm)
+// |p| >= eps decided as re^2 + im^2 >= eps^2 in double: both squares are exact there and the
+// sum rounds once, so the decision is reproducible bit for bit.  The fp32 sum of squares is
+// within 2^-22 of the exact one, so it settles every case outside a 2^-21 band around the
+// threshold; only the band takes the double path.
+__device__ __forceinline__ bool gate_open(float re, float im, const ScanParams &prm)
+{
+    const float s = fmaf(re, re, im * im);
+    bool open = s >= prm.gate_hi;
+    if (!open && s >= prm.gate_lo)
+        open = ((double)re * (double)re + (double)im * (double)im >= prm.eps2);
+    return open;
+}
+
+template <int T, int W, int KIND, bool VEC, bool FULL>
+__device__ __forceinline__ void scan_tile(const ScanParams &prm, float4 (*sE)[32], float4 (*sR)[32],
+                                          float (*sCoef)[6], unsigned long long *sEpoch, int *sErr,
+                                          const int g, const int b, const int k)
 {
     constexpr bool REV = (KIND == KIND_BWD);
     constexpr int TILE = T * W;
-    __shared__ float4 sE[W][32];
-    __shared__ float sCoef[64][6];
-    __shared__ float4 sS[32];
-    __shared__ int sErr;
-
+    constexpr int M = W - 1;
     const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
-    const int G = prm.G, B = prm.B, C = prm.C, K = prm.K;
+    const int G = prm.G, C = prm.C, K = prm.K;
     const long long L = prm.L;
-    const int g = blockIdx.x % G;
-    const int bk = blockIdx.x / G;
-    const int b = bk % B;
-    const int k = bk / B;                         // tile index along (logical) time
-    const int c0 = g * 64 + lane, c1 = c0 + 32;
-    const bool v0 = c0 < C, v1 = c1 < C;
+    const int c0 = g * 64 + 2 * lane;
+    const bool vA = FULL || c0 < C, vB = FULL || c0 + 1 < C;
     const long long s0 = (long long)k * TILE + (long long)w * T;   // first logical step
-    const long long rem = L - s0;
-    const int nvalid = rem <= 0 ? 0 : (rem >= T ? T : (int)rem);
+    int nvalid = T;
+    if (!FULL) {
+        const long long rem = L - s0;
+        nvalid = rem <= 0 ? 0 : (rem >= T ? T : (int)rem);
+    }
     // logical step s <-> physical row t: forward t = s, reverse t = L-1-s
     const long long t_first = REV ? (L - 1 - s0) : s0;
     const long long rowstep = REV ? -(long long)C : (long long)C;
-    const long long row0 = ((long long)b * L + t_first) * C;       // only used when nvalid > 0
-
-    unsigned long long epoch = 0;
-    if (w == 0) epoch = ld_volatile_u64(&prm.ws->epoch);
-    if (tid == 0) sErr = 0;
+    const long long e0 = ((long long)b * L + t_first) * C + c0;    // only used when nvalid > 0
 
     // ---- 0. loads -------------------------------------------------------------------------
-    float2 x0[T], x1[T];
+    float4 x[T];
     {
-        const float2 *in = reinterpret_cast<const float2 *>(prm.in);
+        const float2 *in = reinterpret_cast<const float2 *>(prm.in) + e0;
 #pragma unroll
         for (int i = 0; i < T; ++i) {
-            x0[i] = make_float2(0.f, 0.f);
-            x1[i] = make_float2(0.f, 0.f);
-            if (i < nvalid) {
-                const float2 *r = in + row0 + (long long)i * rowstep;
-                if (v0) x0[i] = __ldcs(r + c0);
-                if (v1) x1[i] = __ldcs(r + c1);
+            x[i] = zero4();
+            if (FULL || i < nvalid) {
+                const float2 *r = in + (long long)i * rowstep;
+                if (VEC) {
+                    if (vA) x[i] = __ldcs(reinterpret_cast<const float4 *>(r));
+                } else {
+                    if (vA) { const float2 v = __ldcs(r); x[i].x = v.x; x[i].y = v.y; }
+                    if (vB) { const float2 v = __ldcs(r + 1); x[i].z = v.x; x[i].w = v.y; }
+                }
             }
         }
     }
-    float2 q0[KIND == KIND_BWD ? T : 1], q1[KIND == KIND_BWD ? T : 1];   // P_{t-1}
+    float4 q[KIND == KIND_BWD ? T : 1];                            // P_{t-1}
     if constexpr (KIND == KIND_BWD) {
-        const float2 *aux = reinterpret_cast<const float2 *>(prm.aux);
 #pragma unroll
         for (int i = 0; i < T; ++i) {
-            q0[i] = make_float2(0.f, 0.f);
-            q1[i] = make_float2(0.f, 0.f);
-            if (aux != nullptr && i < nvalid) {
+            q[i] = zero4();
+            if (prm.aux != nullptr && (FULL || i < nvalid)) {
                 const long long t = t_first - i;
                 if (t >= 1) {
-                    const float2 *r = aux + ((long long)b * L + t - 1) * C;
-                    if (v0) q0[i] = __ldcs(r + c0);
-                    if (v1) q1[i] = __ldcs(r + c1);
+                    const float2 *r = reinterpret_cast<const float2 *>(prm.aux) + e0 - C + (long long)i * rowstep;
+                    if (VEC) {
+                        if (vA) q[i] = __ldcs(reinterpret_cast<const float4 *>(r));
+                    } else {
+                        if (vA) { const float2 v = __ldcs(r); q[i].x = v.x; q[i].y = v.y; }
+                        if (vB) { const float2 v = __ldcs(r + 1); q[i].z = v.x; q[i].w = v.y; }
+                    }
                 } else if (prm.state_in != nullptr) {
-                    if (v0) q0[i] = prm.state_in[(long long)b * C + c0];
-                    if (v1) q1[i] = prm.state_in[(long long)b * C + c1];
+                    const float2 *r = prm.state_in + (long long)b * C + c0;
+                    if (vA) { const float2 v = r[0]; q[i].x = v.x; q[i].y = v.y; }
+                    if (vB) { const float2 v = r[1]; q[i].z = v.x; q[i].w = v.y; }
                 }
             }
         }
         // lam_{L-1} = G_{L-1} + grad_state_out: fold it into the first logical step
         if (prm.edge_in != nullptr && s0 == 0 && nvalid > 0) {
-            if (v0) { const float2 e = prm.edge_in[(long long)b * C + c0]; x0[0].x += e.x; x0[0].y += e.y; }
-            if (v1) { const float2 e = prm.edge_in[(long long)b * C + c1]; x1[0].x += e.x; x1[0].y += e.y; }
+            const float2 *r = prm.edge_in + (long long)b * C + c0;
+            if (vA) { const float2 v = r[0]; x[0].x += v.x; x[0].y += v.y; }
+            if (vB) { const float2 v = r[1]; x[0].z += v.x; x[0].w += v.y; }
         }
     }
 
@@ -137,134 +161,146 @@ __global__ void __launch_bounds__(W * 32) cawn_scan_kernel(const ScanParams prm)
 #pragma unroll
         for (int i = 0; i < 6; ++i) sCoef[tid][i] = cf[i];
     }
-    __syncthreads();
-    const float2 a0 = make_float2(sCoef[lane][0], sCoef[lane][1]);
-    const float2 a1 = make_float2(sCoef[lane + 32][0], sCoef[lane + 32][1]);
-    const float2 aT0 = make_float2(sCoef[lane][2], sCoef[lane][3]);
-    const float2 aT1 = make_float2(sCoef[lane + 32][2], sCoef[lane + 32][3]);
+    unsigned long long epoch0 = 0;
+    unsigned arrived = 0;
+    if (tid == 0) {
+        epoch0 = ld_volatile_u64(&prm.ws->epoch);
+        *sEpoch = epoch0;
+        *sErr = 0;
+        // counted only once the epoch has been read (the increment depends on its value)
+        arrived = atomicAdd(&prm.ws->done, 1u + (unsigned)(epoch0 >> 63));
+    }
+    __syncthreads();                                                           // barrier 1
+    float4 a, aT;
+    {
+        // channel 2l: a, a^T, A at sCoef[2l][0..5]; channel 2l+1 follows: 12 contiguous floats
+        const float4 *cp = reinterpret_cast<const float4 *>(&sCoef[2 * lane][0]);
+        const float4 u0 = cp[0], u1 = cp[1], u2 = cp[2];
+        a = make_float4(u0.x, u0.y, u1.z, u1.w);
+        aT = make_float4(u0.z, u0.w, u2.x, u2.y);
+    }
+    const unsigned long long epoch = *sEpoch;
 
     // ---- 1. gate + local reduction from a zero start ---------------------------------------
-    float2 e0 = make_float2(0.f, 0.f), e1 = e0;
+    float4 e = zero4();
 #pragma unroll
     for (int i = 0; i < T; ++i) {
         if constexpr (KIND == KIND_FWD) {
-            // |p| >= eps decided as re^2 + im^2 >= eps^2 in double: both squares are exact
-            // there and the sum rounds once, so the mask is reproducible bit for bit.
-            const bool o0 = v0 && ((double)x0[i].x * (double)x0[i].x +
-                                   (double)x0[i].y * (double)x0[i].y >= prm.eps2);
-            const bool o1 = v1 && ((double)x1[i].x * (double)x1[i].x +
-                                   (double)x1[i].y * (double)x1[i].y >= prm.eps2);
-            if (!o0) x0[i] = make_float2(0.f, 0.f);
-            if (!o1) x1[i] = make_float2(0.f, 0.f);
+            const bool oA = vA && gate_open(x[i].x, x[i].y, prm);
+            const bool oB = vB && gate_open(x[i].z, x[i].w, prm);
+            if (!oA) { x[i].x = 0.f; x[i].y = 0.f; }
+            if (!oB) { x[i].z = 0.f; x[i].w = 0.f; }
             if (prm.mask != nullptr) {
-                const unsigned m0 = __ballot_sync(0xffffffffu, o0);
-                const unsigned m1 = __ballot_sync(0xffffffffu, o1);
-                if (lane == 0 && i < nvalid) {
+                // lanes 0..15 hold channels 0..31 of the group (word 0), lanes 16..31 word 1
+                const unsigned bits = ((oA ? 1u : 0u) | (oB ? 2u : 0u)) << (2 * (lane & 15));
+                const unsigned w0 = __reduce_or_sync(0xffffffffu, lane < 16 ? bits : 0u);
+                const unsigned w1 = __reduce_or_sync(0xffffffffu, lane < 16 ? 0u : bits);
+                if (FULL || i < nvalid) {
                     uint32_t *mrow = prm.mask + ((long long)b * L + (s0 + i)) * prm.MW + g * 2;
-                    mrow[0] = m0;
-                    if (g * 2 + 1 < prm.MW) mrow[1] = m1;
+                    if (lane == 0) mrow[0] = w0;
+                    if (lane == 16 && g * 2 + 1 < prm.MW) mrow[1] = w1;
                 }
             }
         }
-        if (i < nvalid) {
-            e0 = cfma(a0, e0, x0[i]);
-            e1 = cfma(a1, e1, x1[i]);
-        }
+        if (FULL || i < nvalid) e = cfma2(a, e, x[i]);
     }
-    sE[w][lane] = make_float4(e0.x, e0.y, e1.x, e1.y);
-    __syncthreads();
+    sE[w][lane] = e;
+    if (tid == 0 && arrived == gridDim.x - 1) {
+        // every CTA of this launch has read the epoch: open the next one
+        st_volatile_u32(&prm.ws->done, 0u);
+        st_volatile_u64(&prm.ws->epoch, epoch0 + 1ull);
+    }
+    __syncthreads();                                                           // barrier 2
 
-    // ---- 2. tile aggregate, look-back, inclusive prefix (warp 0) ----------------------------
-    if (w == 0) {
-        const float2 aW0 = make_float2(sCoef[lane][4], sCoef[lane][5]);
-        const float2 aW1 = make_float2(sCoef[lane + 32][4], sCoef[lane + 32][5]);
-        float4 v = sE[0][lane];
-        float2 E0 = make_float2(v.x, v.y), E1 = make_float2(v.z, v.w);
+    // ---- 2. publish the aggregate, fetch the carry window ----------------------------------
+    const long long chain = (long long)b * G + g;
+    const int cpt = k > 0 ? M * ((k - 1) / M) : 0;       // last checkpoint before this tile
+    const int nrec = k - cpt;                            // aggregates in the window, 0..M
+    if (w == 0 && k + 1 < K) {
+        float4 E = sE[0][lane];
 #pragma unroll
-        for (int i = 1; i < W; ++i) {
-            v = sE[i][lane];
-            E0 = cfma(aT0, E0, make_float2(v.x, v.y));
-            E1 = cfma(aT1, E1, make_float2(v.z, v.w));
-        }
-        float2 S0 = make_float2(0.f, 0.f), S1 = S0;
+        for (int i = 1; i < W; ++i) E = cfma2(aT, E, sE[i][lane]);
+        publish_pair(prm.agg + (chain * K + k) * 64, lane, E, epoch, REC_AGGREGATE);
+    }
+    {
+        float4 r = zero4();
         bool ok = true;
-        uint4 *chain = prm.rec + ((long long)(b * G + g) * K) * 64;
-        uint4 *mine = chain + (long long)k * 64;
-        const bool publish = (k + 1 < K);
-        if (k == 0) {
-            if (!REV && prm.state_in != nullptr) {
-                if (v0) S0 = prm.state_in[(long long)b * C + c0];
-                if (v1) S1 = prm.state_in[(long long)b * C + c1];
+        if (w < nrec) {
+            ok = poll_pair(prm.agg + (chain * K + (k - 1 - w)) * 64, lane, epoch, prm.poll_limit, r);
+        } else if (w == W - 1) {
+            if (cpt > 0) {
+                ok = poll_pair(prm.pre + (chain * prm.KP + cpt / M) * 64, lane, epoch, prm.poll_limit, r);
+            } else if (!REV && prm.state_in != nullptr) {
+                const float2 *s = prm.state_in + (long long)b * C + c0;
+                if (vA) { const float2 v = s[0]; r.x = v.x; r.y = v.y; }
+                if (vB) { const float2 v = s[1]; r.z = v.x; r.w = v.y; }
             }
-        } else {
-            if (publish) {
-                st_record(mine + lane, E0, epoch * 4ull + REC_AGGREGATE);
-                st_record(mine + lane + 32, E1, epoch * 4ull + REC_AGGREGATE);
-            }
-            ok = carry_lookback(chain, k, lane, v0, v1, epoch, aW0, aW1, prm.poll_limit, S0, S1);
-            ok = __all_sync(0xffffffffu, ok);
         }
-        if (publish) {
-            const unsigned kind = ok ? REC_PREFIX : REC_POISON;
-            st_record(mine + lane, cfma(aW0, S0, E0), epoch * 4ull + kind);
-            st_record(mine + lane + 32, cfma(aW1, S1, E1), epoch * 4ull + kind);
+        sR[w][lane] = r;
+        if (!ok) {
+            *sErr = 1;
+            atomicMax(&prm.ws->status, 1u);              // CAWN_ERR_CARRY_TIMEOUT
         }
-        if (!ok && lane == 0) {
-            sErr = 1;
-            atomicMax(&prm.ws->status, 1u);          // CAWN_ERR_CARRY_TIMEOUT
-        }
-        sS[lane] = make_float4(S0.x, S0.y, S1.x, S1.y);
     }
-    __syncthreads();
+    __syncthreads();                                                           // barrier 3
 
-    // ---- 3. carry-in of this thread, the recurrence itself, stores --------------------------
-    float2 qa0 = make_float2(0.f, 0.f), qa1 = qa0;
-    if (sErr == 0) {
-        const float4 sv = sS[lane];
-        float2 P0 = make_float2(sv.x, sv.y), P1 = make_float2(sv.z, sv.w);
+    // ---- 3. carry-in, the recurrence itself, stores -----------------------------------------
+    const bool failed = (*sErr != 0);
+    const bool checkpoint = (k > 0 && k % M == 0 && k + 1 < K);
+    float4 qa = zero4();
+    if (!failed) {
+        float4 P = sR[W - 1][lane];
+        {
+            const float4 *cp = reinterpret_cast<const float4 *>(&sCoef[2 * lane][0]);
+            const float4 u1 = cp[1], u2 = cp[2];
+            const float4 AA = make_float4(u1.x, u1.y, u2.z, u2.w);
 #pragma unroll
-        for (int i = 0; i < W - 1; ++i) {
-            if (i < w) {
-                const float4 v = sE[i][lane];
-                P0 = cfma(aT0, P0, make_float2(v.x, v.y));
-                P1 = cfma(aT1, P1, make_float2(v.z, v.w));
-            }
+            for (int i = M - 1; i >= 0; --i)
+                if (i < nrec) P = cfma2(AA, P, sR[i][lane]);
         }
-        float2 *out = reinterpret_cast<float2 *>(prm.out);
+        if (checkpoint && w == 0)
+            publish_pair(prm.pre + (chain * prm.KP + k / M) * 64, lane, P, epoch, REC_PREFIX);
+#pragma unroll
+        for (int i = 0; i < W - 1; ++i)
+            if (i < w) P = cfma2(aT, P, sE[i][lane]);
+
+        float2 *out = reinterpret_cast<float2 *>(prm.out) + e0;
         const float cl = prm.clampv;
 #pragma unroll
         for (int i = 0; i < T; ++i) {
-            if (i < nvalid) {
-                P0 = cfma(a0, P0, x0[i]);
-                P1 = cfma(a1, P1, x1[i]);
-                float2 o0 = P0, o1 = P1;
-                if (cl > 0.f) {
-                    o0.x = clampf(o0.x, cl); o0.y = clampf(o0.y, cl);
-                    o1.x = clampf(o1.x, cl); o1.y = clampf(o1.y, cl);
+            if (FULL || i < nvalid) {
+                P = cfma2(a, P, x[i]);
+                const float4 o = cl > 0.f ? clamp4(P, cl) : P;
+                float2 *r = out + (long long)i * rowstep;
+                if (VEC) {
+                    if (vA) __stcs(reinterpret_cast<float4 *>(r), o);
+                } else {
+                    if (vA) __stcs(r, make_float2(o.x, o.y));
+                    if (vB) __stcs(r + 1, make_float2(o.z, o.w));
                 }
-                float2 *r = out + row0 + (long long)i * rowstep;
-                if (v0) __stcs(r + c0, o0);
-                if (v1) __stcs(r + c1, o1);
                 if constexpr (KIND == KIND_BWD) {
                     // conj(lam) * P_{t-1}
-                    qa0.x = fmaf(P0.x, q0[i].x, fmaf(P0.y, q0[i].y, qa0.x));
-                    qa0.y = fmaf(P0.x, q0[i].y, fmaf(-P0.y, q0[i].x, qa0.y));
-                    qa1.x = fmaf(P1.x, q1[i].x, fmaf(P1.y, q1[i].y, qa1.x));
-                    qa1.y = fmaf(P1.x, q1[i].y, fmaf(-P1.y, q1[i].x, qa1.y));
+                    qa.x = fmaf(P.x, q[i].x, fmaf(P.y, q[i].y, qa.x));
+                    qa.y = fmaf(P.x, q[i].y, fmaf(-P.y, q[i].x, qa.y));
+                    qa.z = fmaf(P.z, q[i].z, fmaf(P.w, q[i].w, qa.z));
+                    qa.w = fmaf(P.z, q[i].w, fmaf(-P.w, q[i].z, qa.w));
                 }
             }
         }
         // the thread that owns the last step writes the carried state (never clamped)
         if (prm.state_out != nullptr && nvalid > 0 && s0 + nvalid == L) {
-            if (REV) { P0 = cmul(a0, P0); P1 = cmul(a1, P1); }   // grad_state_in = conj(a) lam_0
-            if (v0) prm.state_out[(long long)b * C + c0] = P0;
-            if (v1) prm.state_out[(long long)b * C + c1] = P1;
+            if (REV) P = cmul2(a, P);                    // grad_state_in = conj(a) lam_0
+            float2 *s = prm.state_out + (long long)b * C + c0;
+            if (vA) s[0] = make_float2(P.x, P.y);
+            if (vB) s[1] = make_float2(P.z, P.w);
         }
+    } else if (checkpoint && w == 0) {
+        publish_pair(prm.pre + (chain * prm.KP + k / M) * 64, lane, zero4(), epoch, REC_POISON);
     }
     if constexpr (KIND == KIND_BWD) {
         if (prm.qpart != nullptr) {
             __syncthreads();
-            sE[w][lane] = make_float4(qa0.x, qa0.y, qa1.x, qa1.y);
+            sE[w][lane] = qa;
             __syncthreads();
             if (w == 0) {
                 float4 acc = sE[0][lane];
@@ -273,21 +309,31 @@ __global__ void __launch_bounds__(W * 32) cawn_scan_kernel(const ScanParams prm)
                     const float4 v = sE[i][lane];
                     acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
                 }
-                float2 *qp = prm.qpart + ((long long)b * K + k) * C;
-                if (v0) qp[c0] = make_float2(acc.x, acc.y);
-                if (v1) qp[c1] = make_float2(acc.z, acc.w);
+                float2 *qp = prm.qpart + ((long long)b * K + k) * C + c0;
+                if (vA) qp[0] = make_float2(acc.x, acc.y);
+                if (vB) qp[1] = make_float2(acc.z, acc.w);
             }
         }
     }
+}
 
-    // ---- launch bookkeeping: the last CTA opens the next epoch ------------------------------
-    if (tid == 0) {
-        const unsigned prev = atomicAdd(&prm.ws->done, 1u);
-        if (prev == gridDim.x - 1) {
-            prm.ws->done = 0;
-            st_volatile_u64(&prm.ws->epoch, epoch + 1ull);
-        }
-    }
+template <int T, int W, int KIND, bool VEC>
+__global__ void __launch_bounds__(W * 32) cawn_scan_kernel(const ScanParams prm)
+{
+    constexpr int TILE = T * W;
+    __shared__ float4 sE[W][32];
+    __shared__ float4 sR[W][32];
+    __shared__ __align__(16) float sCoef[64][6];
+    __shared__ unsigned long long sEpoch;
+    __shared__ int sErr;
+
+    const int g = blockIdx.x % prm.G;
+    const int bk = blockIdx.x / prm.G;
+    const int b = bk % prm.B;
+    const int k = bk / prm.B;                         // tile index along (logical) time
+    const bool full = ((long long)(k + 1) * TILE <= prm.L) && (g * 64 + 64 <= prm.C);
+    if (full) scan_tile<T, W, KIND, VEC, true>(prm, sE, sR, sCoef, &sEpoch, &sErr, g, b, k);
+    else      scan_tile<T, W, KIND, VEC, false>(prm, sE, sR, sCoef, &sEpoch, &sErr, g, b, k);
 }
 
 // grad_gamma_j = Re(e^{i theta} Q_j), grad_theta_j = -Im(a_j Q_j), Q_j = sum of the per-tile

@@ -45,8 +45,9 @@ def test_workspace_sizes_are_host_only_and_monotone():
     small = cb.cawn_workspace_bytes(cb.make_params(1, 256, 4, 16), cb.CAWN_OP_FWD)
     big = cb.cawn_workspace_bytes(cb.make_params(8, 2048, 12, 64), cb.CAWN_OP_FWD)
     assert 256 < small < big
-    # tile = 128 steps, 64-channel groups, 64 records of 16 B per (batch, group, tile)
-    assert big == 256 + 8 * 12 * 16 * 64 * 16
+    # tile = 128 steps, 64-channel groups; per (batch, group): one 64 x 16 B aggregate record per
+    # tile (16) plus one checkpoint record per 7 tiles (16 // 7 + 1 = 3 slots)
+    assert big == 256 + 8 * 12 * (16 + 3) * 64 * 16
     st = cb.cawn_workspace_bytes(cb.make_params(2, 10, 12, 64, conv_k=4), cb.CAWN_OP_STATE)
     assert st == 2 * 768 * 8 + 2 * 3 * 768 * 4
     saved = cb.cawn_workspace_bytes(cb.make_params(8, 4096, 12, 64), cb.CAWN_OP_BWD_SAVED)
