@@ -95,22 +95,42 @@ inline bool grid_ok(const cawn_params *p, const Geometry &g)
 }
 
 // The float4 path needs every row segment on a 16-byte boundary: C even (the arrays
-// themselves are checked to be 16-byte aligned).
-template <int T, int W, int KIND>
-cudaError_t launch_scan(const ScanParams &sp, cudaStream_t st)
+// themselves are checked to be 16-byte aligned).  The tile is staged in dynamic shared memory;
+// MINB is the number of CTAs per SM the register allocation leaves room for.
+template <int T, int W, int KIND, bool VEC, int MINB>
+cudaError_t launch_scan_inst(const ScanParams &sp, cudaStream_t st)
 {
+    constexpr size_t smem = sizeof(ScanSmem<T, W, KIND>);
+    static bool configured[64] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64 || !configured[dev]) {
+        e = cudaFuncSetAttribute(cawn_scan_kernel<T, W, KIND, VEC, MINB>,
+                                 cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        if (dev >= 0 && dev < 64) configured[dev] = true;
+    }
     const unsigned grid = (unsigned)((long long)sp.B * sp.G * sp.K);
-    if (sp.C % 2 == 0) cawn_scan_kernel<T, W, KIND, true><<<grid, W * 32, 0, st>>>(sp);
-    else               cawn_scan_kernel<T, W, KIND, false><<<grid, W * 32, 0, st>>>(sp);
+    cawn_scan_kernel<T, W, KIND, VEC, MINB><<<grid, W * 32, smem, st>>>(sp);
     return cudaGetLastError();
 }
-
-template <int KIND>
-cudaError_t launch_scan_shape(TileShape ts, const ScanParams &sp, cudaStream_t st)
+template <int T, int W, int KIND, int MINB>
+cudaError_t launch_scan(const ScanParams &sp, cudaStream_t st)
 {
-    if (ts.T == 16 && ts.W == 8) return launch_scan<16, 8, KIND>(sp, st);
-    if (ts.T == 8 && ts.W == 8) return launch_scan<8, 8, KIND>(sp, st);
-    return launch_scan<4, 4, KIND>(sp, st);
+    return sp.C % 2 == 0 ? launch_scan_inst<T, W, KIND, true, MINB>(sp, st)
+                         : launch_scan_inst<T, W, KIND, false, MINB>(sp, st);
+}
+
+inline cudaError_t launch_fwd(TileShape ts, const ScanParams &sp, cudaStream_t st)
+{
+    if (ts.T == 16) return launch_scan<16, 8, KIND_FWD, 3>(sp, st);
+    return launch_scan<4, 4, KIND_FWD, 8>(sp, st);
+}
+inline cudaError_t launch_bwd(TileShape ts, const ScanParams &sp, cudaStream_t st)
+{
+    if (ts.T == 8) return launch_scan<8, 8, KIND_BWD, 3>(sp, st);
+    return launch_scan<4, 4, KIND_BWD, 8>(sp, st);
 }
 
 // Host-staged forward: layout of the device scratch.
@@ -244,7 +264,7 @@ int cawn_phase_accumulate_fwd(const cawn_params *params, const void *input,
     set_gate(sp, params->gate_eps);
     sp.clampv = params->clamp_abs > 0.f ? params->clamp_abs : 0.f;
     sp.poll_limit = kPollLimit;
-    if (launch_scan_shape<KIND_FWD>(ts, sp, st) != cudaSuccess) return CAWN_ERR_CUDA;
+    if (launch_fwd(ts, sp, st) != cudaSuccess) return CAWN_ERR_CUDA;
     return CAWN_OK;
 }
 
@@ -310,7 +330,7 @@ int cawn_phase_accumulate_bwd(const cawn_params *params, const void *saved, int 
         set_gate(fp, params->gate_eps);
         fp.clampv = 0.f;
         fp.poll_limit = kPollLimit;
-        if (launch_scan_shape<KIND_FWD>(tf, fp, st) != cudaSuccess) return CAWN_ERR_CUDA;
+        if (launch_fwd(tf, fp, st) != cudaSuccess) return CAWN_ERR_CUDA;
         states = Pbuf;
     }
 
@@ -328,7 +348,7 @@ int cawn_phase_accumulate_bwd(const cawn_params *params, const void *saved, int 
     sp.L = params->L; sp.B = params->B;
     sp.clampv = params->grad_clamp_abs > 0.f ? params->grad_clamp_abs : 0.f;
     sp.poll_limit = kPollLimit;
-    if (launch_scan_shape<KIND_BWD>(tb, sp, st) != cudaSuccess) return CAWN_ERR_CUDA;
+    if (launch_bwd(tb, sp, st) != cudaSuccess) return CAWN_ERR_CUDA;
 
     if (want_param) {
         const int warps = 8;

@@ -3,16 +3,21 @@
 // One CTA owns a tile of TILE = W*T consecutive time steps of one (batch, 64-channel group).
 // Warp w owns T consecutive steps; lane l owns the adjacent channels 64g + 2l and 64g + 2l + 1,
 // so a warp-wide access is one 512-byte row segment read or written as 32 float4.
-// The tile lives in registers between its single read and its single write:
+// The tile is staged in shared memory between its single read from and its single write to
+// global memory: the asynchronous copies hold no registers while they are in flight, which
+// is what lets three 64 KB tiles per SM stay in flight next to the arithmetic.
 //
-//   0. every thread issues all of its loads (T rows, independent); meanwhile 64 threads
-//      prepare the per-channel coefficients a, a^T, a^TILE in double            [barrier 1]
-//   1. gate (Cartesian forward), then each thread reduces its T steps from a zero start and
-//      leaves the end state in shared memory                                     [barrier 2]
+//   0. every thread issues the asynchronous copies of its own T row pieces; meanwhile 64
+//      threads prepare the per-channel coefficients a, a^T, a^TILE in double     [barrier 1]
+//   1. gate (Cartesian forward; the gated value goes back to shared memory), and each thread
+//      reduces its T steps from a zero start, leaving the end state in shared memory
+//                                                                                [barrier 2]
 //   2. warp 0 folds the W ends into the tile aggregate and publishes it; then every warp
 //      fetches one record of the carry window (below) into shared memory         [barrier 3]
 //   3. every warp folds the window into the tile's carry-in, folds the earlier warps' ends on
 //      top, re-runs its T steps as the plain recurrence from that state and stores them
+//
+// A thread only ever touches the tile rows it copied itself, so the tile needs no barrier.
 //
 // Carry window.  With M = W-1, the tiles k = M, 2M, ... of a chain are checkpoints: they also
 // publish their carry-in X_k (the state before the tile).  Tile k reads the carry-in of the
@@ -57,22 +62,47 @@ struct ScanParams {
     unsigned poll_limit;
 };
 
-// |p| >= eps decided as re^2 + im^2 >= eps^2 in double: both squares are exact there and the
-// sum rounds once, so the decision is reproducible bit for bit.  The fp32 sum of squares is
-// within 2^-22 of the exact one, so it settles every case outside a 2^-21 band around the
-// threshold; only the band takes the double path.
-__device__ __forceinline__ bool gate_open(float re, float im, const ScanParams &prm)
+// Shared memory of one CTA: the tile (two tiles in the backward: grad_y and P_{t-1}), then the
+// small exchange areas.
+template <int T, int W, int KIND>
+struct ScanSmem {
+    static constexpr int TILE = T * W;
+    static constexpr int NT = (KIND == KIND_BWD) ? 2 : 1;
+    float4 tile[NT][TILE][32];
+    float4 sE[W][32];
+    float4 sR[W][32];
+    float sCoef[64][6];
+    unsigned long long epoch;
+    int err;
+    int pad;
+};
+
+__device__ __forceinline__ uint32_t smem_addr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void cp_async16(void *dst, const void *src)
 {
-    const float s = fmaf(re, re, im * im);
-    bool open = s >= prm.gate_hi;
-    if (!open && s >= prm.gate_lo)
-        open = ((double)re * (double)re + (double)im * (double)im >= prm.eps2);
-    return open;
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"(smem_addr(dst)), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async8(void *dst, const void *src)
+{
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" :: "r"(smem_addr(dst)), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+
+// Copy (asynchronously) or zero one row piece of this lane: two adjacent complex64.
+template <bool VEC>
+__device__ __forceinline__ void fetch_piece(float4 *dst, const float2 *src, bool vA, bool vB)
+{
+    if (VEC) {
+        if (vA) cp_async16(dst, src); else *dst = zero4();
+    } else {
+        float2 *d = reinterpret_cast<float2 *>(dst);
+        if (vA) cp_async8(d, src); else d[0] = make_float2(0.f, 0.f);
+        if (vB) cp_async8(d + 1, src + 1); else d[1] = make_float2(0.f, 0.f);
+    }
 }
 
 template <int T, int W, int KIND, bool VEC, bool FULL>
-__device__ __forceinline__ void scan_tile(const ScanParams &prm, float4 (*sE)[32], float4 (*sR)[32],
-                                          float (*sCoef)[6], unsigned long long *sEpoch, int *sErr,
+__device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, KIND> &sm,
                                           const int g, const int b, const int k)
 {
     constexpr bool REV = (KIND == KIND_BWD);
@@ -91,54 +121,29 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, float4 (*sE)[32
     }
     // logical step s <-> physical row t: forward t = s, reverse t = L-1-s
     const long long t_first = REV ? (L - 1 - s0) : s0;
-    const long long rowstep = REV ? -(long long)C : (long long)C;
+    const long long rowstep = REV ? -(long long)C : (long long)C;  // in complex elements
     const long long e0 = ((long long)b * L + t_first) * C + c0;    // only used when nvalid > 0
+    float4 *const xs = &sm.tile[0][w * T][lane];                   // this thread's pieces, 32 float4 apart
 
-    // ---- 0. loads -------------------------------------------------------------------------
-    float4 x[T];
+    // ---- 0. asynchronous copies into shared memory -----------------------------------------
     {
-        const float2 *in = reinterpret_cast<const float2 *>(prm.in) + e0;
+        const float2 *r = reinterpret_cast<const float2 *>(prm.in) + e0;
 #pragma unroll
         for (int i = 0; i < T; ++i) {
-            x[i] = zero4();
-            if (FULL || i < nvalid) {
-                const float2 *r = in + (long long)i * rowstep;
-                if (VEC) {
-                    if (vA) x[i] = __ldcs(reinterpret_cast<const float4 *>(r));
-                } else {
-                    if (vA) { const float2 v = __ldcs(r); x[i].x = v.x; x[i].y = v.y; }
-                    if (vB) { const float2 v = __ldcs(r + 1); x[i].z = v.x; x[i].w = v.y; }
-                }
-            }
+            const bool row = FULL || i < nvalid;
+            fetch_piece<VEC>(xs + i * 32, r, row && vA, row && vB);
+            r += rowstep;
         }
     }
-    float4 q[KIND == KIND_BWD ? T : 1];                            // P_{t-1}
     if constexpr (KIND == KIND_BWD) {
+        float4 *const qs = &sm.tile[1][w * T][lane];
+        const bool have = prm.aux != nullptr;
+        const float2 *r = reinterpret_cast<const float2 *>(prm.aux) + e0 - C;   // row t-1
 #pragma unroll
         for (int i = 0; i < T; ++i) {
-            q[i] = zero4();
-            if (prm.aux != nullptr && (FULL || i < nvalid)) {
-                const long long t = t_first - i;
-                if (t >= 1) {
-                    const float2 *r = reinterpret_cast<const float2 *>(prm.aux) + e0 - C + (long long)i * rowstep;
-                    if (VEC) {
-                        if (vA) q[i] = __ldcs(reinterpret_cast<const float4 *>(r));
-                    } else {
-                        if (vA) { const float2 v = __ldcs(r); q[i].x = v.x; q[i].y = v.y; }
-                        if (vB) { const float2 v = __ldcs(r + 1); q[i].z = v.x; q[i].w = v.y; }
-                    }
-                } else if (prm.state_in != nullptr) {
-                    const float2 *r = prm.state_in + (long long)b * C + c0;
-                    if (vA) { const float2 v = r[0]; q[i].x = v.x; q[i].y = v.y; }
-                    if (vB) { const float2 v = r[1]; q[i].z = v.x; q[i].w = v.y; }
-                }
-            }
-        }
-        // lam_{L-1} = G_{L-1} + grad_state_out: fold it into the first logical step
-        if (prm.edge_in != nullptr && s0 == 0 && nvalid > 0) {
-            const float2 *r = prm.edge_in + (long long)b * C + c0;
-            if (vA) { const float2 v = r[0]; x[0].x += v.x; x[0].y += v.y; }
-            if (vB) { const float2 v = r[1]; x[0].z += v.x; x[0].w += v.y; }
+            const bool row = have && (FULL || i < nvalid) && (t_first - i >= 1);
+            fetch_piece<VEC>(qs + i * 32, r, row && vA, row && vB);
+            r += rowstep;
         }
     }
 
@@ -159,14 +164,14 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, float4 (*sE)[32
             cf[4] = (float)wr; cf[5] = (float)wi;
         }
 #pragma unroll
-        for (int i = 0; i < 6; ++i) sCoef[tid][i] = cf[i];
+        for (int i = 0; i < 6; ++i) sm.sCoef[tid][i] = cf[i];
     }
     unsigned long long epoch0 = 0;
     unsigned arrived = 0;
     if (tid == 0) {
         epoch0 = ld_volatile_u64(&prm.ws->epoch);
-        *sEpoch = epoch0;
-        *sErr = 0;
+        sm.epoch = epoch0;
+        sm.err = 0;
         // counted only once the epoch has been read (the increment depends on its value)
         arrived = atomicAdd(&prm.ws->done, 1u + (unsigned)(epoch0 >> 63));
     }
@@ -174,37 +179,78 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, float4 (*sE)[32
     float4 a, aT;
     {
         // channel 2l: a, a^T, A at sCoef[2l][0..5]; channel 2l+1 follows: 12 contiguous floats
-        const float4 *cp = reinterpret_cast<const float4 *>(&sCoef[2 * lane][0]);
+        const float4 *cp = reinterpret_cast<const float4 *>(&sm.sCoef[2 * lane][0]);
         const float4 u0 = cp[0], u1 = cp[1], u2 = cp[2];
         a = make_float4(u0.x, u0.y, u1.z, u1.w);
         aT = make_float4(u0.z, u0.w, u2.x, u2.y);
     }
-    const unsigned long long epoch = *sEpoch;
+    const unsigned long long epoch = sm.epoch;
+    cp_async_wait_all();                                  // this thread's pieces have landed
+
+    if constexpr (KIND == KIND_BWD) {
+        // the step at t = 0 multiplies the call's initial state; lam_{L-1} = G_{L-1} + grad_state_out
+        if (nvalid > 0 && t_first - (nvalid - 1) == 0 && prm.aux != nullptr && prm.state_in != nullptr) {
+            const float2 *r = prm.state_in + (long long)b * C + c0;
+            float4 v = zero4();
+            if (vA) { const float2 u = r[0]; v.x = u.x; v.y = u.y; }
+            if (vB) { const float2 u = r[1]; v.z = u.x; v.w = u.y; }
+            sm.tile[1][w * T + (nvalid - 1)][lane] = v;
+        }
+        if (prm.edge_in != nullptr && s0 == 0 && nvalid > 0) {
+            const float2 *r = prm.edge_in + (long long)b * C + c0;
+            float4 v = xs[0];
+            if (vA) { const float2 u = r[0]; v.x += u.x; v.y += u.y; }
+            if (vB) { const float2 u = r[1]; v.z += u.x; v.w += u.y; }
+            xs[0] = v;
+        }
+    }
 
     // ---- 1. gate + local reduction from a zero start ---------------------------------------
     float4 e = zero4();
+    if constexpr (KIND == KIND_FWD) {
+        // |p| >= eps decided as re^2 + im^2 >= eps^2 in double: both squares are exact there
+        // and the sum rounds once, so the decision is reproducible bit for bit.  The fp32 sum
+        // of squares is within 2^-22 of the exact one, so it settles every case outside a
+        // 2^-21 band around the threshold; a row with a lane in the band takes the double path.
+        const float lo = prm.gate_lo, hi = prm.gate_hi;
+        const bool want_mask = prm.mask != nullptr;
+        uint32_t *mrow = prm.mask + ((long long)b * L + s0) * prm.MW + g * 2;
+        const bool second_word = g * 2 + 1 < prm.MW;
 #pragma unroll
-    for (int i = 0; i < T; ++i) {
-        if constexpr (KIND == KIND_FWD) {
-            const bool oA = vA && gate_open(x[i].x, x[i].y, prm);
-            const bool oB = vB && gate_open(x[i].z, x[i].w, prm);
-            if (!oA) { x[i].x = 0.f; x[i].y = 0.f; }
-            if (!oB) { x[i].z = 0.f; x[i].w = 0.f; }
-            if (prm.mask != nullptr) {
+        for (int i = 0; i < T; ++i) {
+            float4 v = xs[i * 32];
+            const float sA = fmaf(v.x, v.x, v.y * v.y), sB = fmaf(v.z, v.z, v.w * v.w);
+            bool oA = sA >= hi, oB = sB >= hi;
+            const bool band = (!oA && sA >= lo) || (!oB && sB >= lo);
+            if (__any_sync(0xffffffffu, band)) {
+                oA = ((double)v.x * (double)v.x + (double)v.y * (double)v.y >= prm.eps2);
+                oB = ((double)v.z * (double)v.z + (double)v.w * (double)v.w >= prm.eps2);
+            }
+            if (!FULL) { oA = oA && vA; oB = oB && vB; }
+            if (!(oA && oB)) {
+                if (!oA) { v.x = 0.f; v.y = 0.f; }
+                if (!oB) { v.z = 0.f; v.w = 0.f; }
+                xs[i * 32] = v;
+            }
+            if (want_mask) {
                 // lanes 0..15 hold channels 0..31 of the group (word 0), lanes 16..31 word 1
                 const unsigned bits = ((oA ? 1u : 0u) | (oB ? 2u : 0u)) << (2 * (lane & 15));
                 const unsigned w0 = __reduce_or_sync(0xffffffffu, lane < 16 ? bits : 0u);
                 const unsigned w1 = __reduce_or_sync(0xffffffffu, lane < 16 ? 0u : bits);
                 if (FULL || i < nvalid) {
-                    uint32_t *mrow = prm.mask + ((long long)b * L + (s0 + i)) * prm.MW + g * 2;
                     if (lane == 0) mrow[0] = w0;
-                    if (lane == 16 && g * 2 + 1 < prm.MW) mrow[1] = w1;
+                    if (lane == 16 && second_word) mrow[1] = w1;
                 }
+                mrow += prm.MW;
             }
+            if (FULL || i < nvalid) e = cfma2(a, e, v);
         }
-        if (FULL || i < nvalid) e = cfma2(a, e, x[i]);
+    } else {
+#pragma unroll
+        for (int i = 0; i < T; ++i)
+            if (FULL || i < nvalid) e = cfma2(a, e, xs[i * 32]);
     }
-    sE[w][lane] = e;
+    sm.sE[w][lane] = e;
     if (tid == 0 && arrived == gridDim.x - 1) {
         // every CTA of this launch has read the epoch: open the next one
         st_volatile_u32(&prm.ws->done, 0u);
@@ -217,9 +263,9 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, float4 (*sE)[32
     const int cpt = k > 0 ? M * ((k - 1) / M) : 0;       // last checkpoint before this tile
     const int nrec = k - cpt;                            // aggregates in the window, 0..M
     if (w == 0 && k + 1 < K) {
-        float4 E = sE[0][lane];
+        float4 E = sm.sE[0][lane];
 #pragma unroll
-        for (int i = 1; i < W; ++i) E = cfma2(aT, E, sE[i][lane]);
+        for (int i = 1; i < W; ++i) E = cfma2(aT, E, sm.sE[i][lane]);
         publish_pair(prm.agg + (chain * K + k) * 64, lane, E, epoch, REC_AGGREGATE);
     }
     {
@@ -236,42 +282,42 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, float4 (*sE)[32
                 if (vB) { const float2 v = s[1]; r.z = v.x; r.w = v.y; }
             }
         }
-        sR[w][lane] = r;
+        sm.sR[w][lane] = r;
         if (!ok) {
-            *sErr = 1;
+            sm.err = 1;
             atomicMax(&prm.ws->status, 1u);              // CAWN_ERR_CARRY_TIMEOUT
         }
     }
     __syncthreads();                                                           // barrier 3
 
     // ---- 3. carry-in, the recurrence itself, stores -----------------------------------------
-    const bool failed = (*sErr != 0);
+    const bool failed = (sm.err != 0);
     const bool checkpoint = (k > 0 && k % M == 0 && k + 1 < K);
     float4 qa = zero4();
     if (!failed) {
-        float4 P = sR[W - 1][lane];
+        float4 P = sm.sR[W - 1][lane];
         {
-            const float4 *cp = reinterpret_cast<const float4 *>(&sCoef[2 * lane][0]);
+            const float4 *cp = reinterpret_cast<const float4 *>(&sm.sCoef[2 * lane][0]);
             const float4 u1 = cp[1], u2 = cp[2];
             const float4 AA = make_float4(u1.x, u1.y, u2.z, u2.w);
 #pragma unroll
             for (int i = M - 1; i >= 0; --i)
-                if (i < nrec) P = cfma2(AA, P, sR[i][lane]);
+                if (i < nrec) P = cfma2(AA, P, sm.sR[i][lane]);
         }
         if (checkpoint && w == 0)
             publish_pair(prm.pre + (chain * prm.KP + k / M) * 64, lane, P, epoch, REC_PREFIX);
 #pragma unroll
         for (int i = 0; i < W - 1; ++i)
-            if (i < w) P = cfma2(aT, P, sE[i][lane]);
+            if (i < w) P = cfma2(aT, P, sm.sE[i][lane]);
 
-        float2 *out = reinterpret_cast<float2 *>(prm.out) + e0;
+        float2 *r = reinterpret_cast<float2 *>(prm.out) + e0;
         const float cl = prm.clampv;
+        const bool clamped = cl > 0.f;
 #pragma unroll
         for (int i = 0; i < T; ++i) {
             if (FULL || i < nvalid) {
-                P = cfma2(a, P, x[i]);
-                const float4 o = cl > 0.f ? clamp4(P, cl) : P;
-                float2 *r = out + (long long)i * rowstep;
+                P = cfma2(a, P, xs[i * 32]);
+                const float4 o = clamped ? clamp4(P, cl) : P;
                 if (VEC) {
                     if (vA) __stcs(reinterpret_cast<float4 *>(r), o);
                 } else {
@@ -280,12 +326,14 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, float4 (*sE)[32
                 }
                 if constexpr (KIND == KIND_BWD) {
                     // conj(lam) * P_{t-1}
-                    qa.x = fmaf(P.x, q[i].x, fmaf(P.y, q[i].y, qa.x));
-                    qa.y = fmaf(P.x, q[i].y, fmaf(-P.y, q[i].x, qa.y));
-                    qa.z = fmaf(P.z, q[i].z, fmaf(P.w, q[i].w, qa.z));
-                    qa.w = fmaf(P.z, q[i].w, fmaf(-P.w, q[i].z, qa.w));
+                    const float4 q = sm.tile[1][w * T + i][lane];
+                    qa.x = fmaf(P.x, q.x, fmaf(P.y, q.y, qa.x));
+                    qa.y = fmaf(P.x, q.y, fmaf(-P.y, q.x, qa.y));
+                    qa.z = fmaf(P.z, q.z, fmaf(P.w, q.w, qa.z));
+                    qa.w = fmaf(P.z, q.w, fmaf(-P.w, q.z, qa.w));
                 }
             }
+            r += rowstep;
         }
         // the thread that owns the last step writes the carried state (never clamped)
         if (prm.state_out != nullptr && nvalid > 0 && s0 + nvalid == L) {
@@ -300,13 +348,13 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, float4 (*sE)[32
     if constexpr (KIND == KIND_BWD) {
         if (prm.qpart != nullptr) {
             __syncthreads();
-            sE[w][lane] = qa;
+            sm.sE[w][lane] = qa;
             __syncthreads();
             if (w == 0) {
-                float4 acc = sE[0][lane];
+                float4 acc = sm.sE[0][lane];
 #pragma unroll
                 for (int i = 1; i < W; ++i) {
-                    const float4 v = sE[i][lane];
+                    const float4 v = sm.sE[i][lane];
                     acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
                 }
                 float2 *qp = prm.qpart + ((long long)b * K + k) * C + c0;
@@ -317,23 +365,20 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, float4 (*sE)[32
     }
 }
 
-template <int T, int W, int KIND, bool VEC>
-__global__ void __launch_bounds__(W * 32) cawn_scan_kernel(const ScanParams prm)
+template <int T, int W, int KIND, bool VEC, int MINB>
+__global__ void __launch_bounds__(W * 32, MINB) cawn_scan_kernel(const ScanParams prm)
 {
     constexpr int TILE = T * W;
-    __shared__ float4 sE[W][32];
-    __shared__ float4 sR[W][32];
-    __shared__ __align__(16) float sCoef[64][6];
-    __shared__ unsigned long long sEpoch;
-    __shared__ int sErr;
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    ScanSmem<T, W, KIND> &sm = *reinterpret_cast<ScanSmem<T, W, KIND> *>(smem_raw);
 
     const int g = blockIdx.x % prm.G;
     const int bk = blockIdx.x / prm.G;
     const int b = bk % prm.B;
     const int k = bk / prm.B;                         // tile index along (logical) time
     const bool full = ((long long)(k + 1) * TILE <= prm.L) && (g * 64 + 64 <= prm.C);
-    if (full) scan_tile<T, W, KIND, VEC, true>(prm, sE, sR, sCoef, &sEpoch, &sErr, g, b, k);
-    else      scan_tile<T, W, KIND, VEC, false>(prm, sE, sR, sCoef, &sEpoch, &sErr, g, b, k);
+    if (full) scan_tile<T, W, KIND, VEC, true>(prm, sm, g, b, k);
+    else      scan_tile<T, W, KIND, VEC, false>(prm, sm, g, b, k);
 }
 
 // grad_gamma_j = Re(e^{i theta} Q_j), grad_theta_j = -Im(a_j Q_j), Q_j = sum of the per-tile
