@@ -20,7 +20,7 @@ struct TileShape { int T, W; };
 inline TileShape fwd_shape(int64_t L) { return L > 32 ? TileShape{16, 8} : TileShape{4, 4}; }
 inline TileShape bwd_shape(int64_t L) { return L > 32 ? TileShape{8, 8} : TileShape{4, 4}; }
 
-// C channels in G groups of 64; K tiles along time, of which every (W-1)-th is a checkpoint
+// C channels in G groups of 64; K tiles along time, of which every kWindow-th is a checkpoint
 // (KP checkpoint slots per chain); MW mask words per row.  Records are 16 bytes per channel.
 struct Geometry {
     int C, G, K, KP, MW;
@@ -34,7 +34,7 @@ inline Geometry geometry(const cawn_params *p, TileShape ts)
     const int64_t tile = (int64_t)ts.T * ts.W;
     g.K = (int)((p->L + tile - 1) / tile);
     if (g.K < 1) g.K = 1;
-    g.KP = g.K / (ts.W - 1) + 1;
+    g.KP = g.K / kWindow + 1;
     g.MW = (g.C + 31) / 32;
     g.agg_bytes = (size_t)p->B * g.G * g.K * 64 * sizeof(uint4);
     g.pre_bytes = (size_t)p->B * g.G * g.KP * 64 * sizeof(uint4);
@@ -50,20 +50,22 @@ inline void set_records(ScanParams &sp, char *rec_base, const Geometry &g)
     sp.G = g.G; sp.K = g.K; sp.KP = g.KP; sp.MW = g.MW; sp.C = g.C;
 }
 
-// fp32 screen of the gate: the fp32 sum of squares is within 2^-22 (relative) of the exact
-// one, so outside a 2^-21 band around eps^2 it already decides the double comparison.
+// fp32 screen of the gate.  The fp32 sum of squares is within 2^-22 (relative) of the exact
+// one, so at a distance of more than 2^-20 eps^2 from fl(eps^2) it already decides the double
+// comparison; inside that band the kernel falls back to double.
 inline void set_gate(ScanParams &sp, float gate_eps)
 {
     const double e2 = (double)gate_eps * (double)gate_eps;
     sp.eps2 = e2;
-    if (e2 == 0.0) {                       // always open (NaN inputs still compare false)
-        sp.gate_lo = 0.f; sp.gate_hi = 0.f;
-    } else if (e2 < 1e-27) {               // fp32 products may be subnormal: screen only far above
-        sp.gate_lo = 0.f; sp.gate_hi = 1e-24f;
+    if (e2 == 0.0) {                       // always open (NaN compares false in either form)
+        sp.gate_mid = 0.f; sp.gate_hw = -1.f; sp.gate_keep = 0.f;
+    } else if (e2 < 1e-27) {               // fp32 squares may be subnormal: keep everything in
+        sp.gate_mid = 0.f; sp.gate_hw = 1e-24f;   // the first pass, decide small sums in double
+        sp.gate_keep = 0.f;
     } else {
-        const double band = 1.0 / 2097152.0;
-        sp.gate_lo = nextafterf((float)(e2 * (1.0 - band)), -INFINITY);
-        sp.gate_hi = nextafterf((float)(e2 * (1.0 + band)), INFINITY);
+        sp.gate_mid = (float)e2;
+        sp.gate_hw = nextafterf((float)(e2 / 1048576.0), INFINITY);
+        sp.gate_keep = -sp.gate_hw;
     }
 }
 
@@ -88,10 +90,10 @@ size_t state_blob_bytes(const cawn_params *p)
     return n;
 }
 
-// Grid size check: tiles are a 1-D grid.
+// Grid size check: tiles are a (G, B, K) grid.
 inline bool grid_ok(const cawn_params *p, const Geometry &g)
 {
-    return (double)p->B * g.G * g.K < 2147483647.0;
+    return p->B <= 65535 && g.K <= 65535 && (double)p->B * g.G * g.K < 4294967295.0;
 }
 
 // The float4 path needs every row segment on a 16-byte boundary: C even (the arrays
@@ -111,7 +113,7 @@ cudaError_t launch_scan_inst(const ScanParams &sp, cudaStream_t st)
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) configured[dev] = true;
     }
-    const unsigned grid = (unsigned)((long long)sp.B * sp.G * sp.K);
+    const dim3 grid((unsigned)sp.G, (unsigned)sp.B, (unsigned)sp.K);
     cawn_scan_kernel<T, W, KIND, VEC, MINB><<<grid, W * 32, smem, st>>>(sp);
     return cudaGetLastError();
 }

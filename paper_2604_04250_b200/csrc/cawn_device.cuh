@@ -119,15 +119,15 @@ __device__ __forceinline__ void publish_pair(uint4 *tile_recs, int lane, float4 
     st_record(tile_recs + 2 * lane + 1, v.z, v.w, tag);
 }
 
-// Wait (with a bound) until both records of this lane's pair carry `epoch`.  Returns false when
-// the wait ran out or the writer published POISON.
+// Wait (with a bound) until both records of this lane's pair carry `epoch`.  (r0, r1) are a
+// first reading taken earlier (zeros if none was taken): if it is already valid no further load
+// is issued.  Returns false when the wait ran out or the writer published POISON.
 __device__ __forceinline__ bool poll_pair(const uint4 *tile_recs, int lane, unsigned long long epoch,
-                                          unsigned poll_limit, float4 &v)
+                                          unsigned poll_limit, uint4 r0, uint4 r1, float4 &v)
 {
     const uint4 *p = tile_recs + 2 * lane;
     unsigned polls = 0;
     for (;;) {
-        const uint4 r0 = ld_record(p), r1 = ld_record(p + 1);
         const unsigned k0 = record_kind(r0, epoch), k1 = record_kind(r1, epoch);
         if (k0 != 0u && k1 != 0u) {
             v = make_float4(__uint_as_float(r0.x), __uint_as_float(r0.y),
@@ -136,6 +136,8 @@ __device__ __forceinline__ bool poll_pair(const uint4 *tile_recs, int lane, unsi
         }
         if (++polls > poll_limit) { v = zero4(); return false; }
         if (polls > 4) __nanosleep(polls > 64 ? 256 : 32);
+        r0 = ld_record(p);
+        r1 = ld_record(p + 1);
     }
 }
 

@@ -7,26 +7,27 @@
 // global memory: the asynchronous copies hold no registers while they are in flight, which
 // is what lets three 64 KB tiles per SM stay in flight next to the arithmetic.
 //
-//   0. every thread issues the asynchronous copies of its own T row pieces; meanwhile 64
-//      threads prepare the per-channel coefficients a, a^T, a^TILE in double     [barrier 1]
-//   1. gate (Cartesian forward; the gated value goes back to shared memory), and each thread
-//      reduces its T steps from a zero start, leaving the end state in shared memory
-//                                                                                [barrier 2]
-//   2. warp 0 folds the W ends into the tile aggregate and publishes it; then every warp
-//      fetches one record of the carry window (below) into shared memory         [barrier 3]
+//   0. every thread issues the asynchronous copies of its own T row pieces, in groups of a few
+//      rows; meanwhile 192 threads prepare the per-channel coefficients a, a^T, a^TILE in
+//      double                                                                    [barrier 1]
+//   1. as its row groups land: gate (Cartesian forward; the gated value goes back to shared
+//      memory), and each thread reduces its T steps from a zero start, leaving the end state
+//      in shared memory                                                          [barrier 2]
+//   2. warp 0 folds the W ends into the tile aggregate and publishes it; every warp fetches
+//      its records of the carry window (below) into shared memory                [barrier 3]
 //   3. every warp folds the window into the tile's carry-in, folds the earlier warps' ends on
 //      top, re-runs its T steps as the plain recurrence from that state and stores them
 //
 // A thread only ever touches the tile rows it copied itself, so the tile needs no barrier.
 //
-// Carry window.  With M = W-1, the tiles k = M, 2M, ... of a chain are checkpoints: they also
+// Carry window.  With M = kWindow, the tiles k = M, 2M, ... of a chain are checkpoints: they also
 // publish their carry-in X_k (the state before the tile).  Tile k reads the carry-in of the
 // last checkpoint c < k (c = 0: the call's initial state) and the aggregates E_c .. E_{k-1},
 // and evaluates X_k = A^(k-c) X_c + sum A^(k-1-i) E_i by Horner's rule, oldest first, A = a^TILE.
 // What is read and the order it is combined in depend on k alone, never on timing, so results
 // are bit-for-bit repeatable; aggregates are published before anything is waited for, so the
 // only serial dependency runs from checkpoint to checkpoint.  A tile only ever waits for tiles
-// with a smaller block index, which the hardware has dispatched before it.
+// with a smaller linear block index, which the hardware has dispatched before it.
 //
 // Each run of the fp32 recurrence is at most T steps long and everything that crosses a thread
 // boundary is multiplied by a power of a_j rounded once from double: the rounding error of
@@ -36,10 +37,14 @@
 // accumulates sum conj(lam_t) P_{t-1} per channel for the retention and rotation gradients.
 #pragma once
 #include "cawn_device.cuh"
+#include <type_traits>
 
 namespace cawn {
 
 enum : int { KIND_FWD = 0, KIND_BWD = 2 };
+
+// Carry window: every kWindow-th tile of a chain is a checkpoint.
+constexpr int kWindow = 7;
 
 struct ScanParams {
     const void *in;              // FWD: pushes p;  BWD: grad_y              [B,L,C] complex64
@@ -57,7 +62,9 @@ struct ScanParams {
     long long L;
     int B, C, G, K, KP, MW;      // MW = mask words per row
     double eps2;                 // gate threshold squared
-    float gate_lo, gate_hi;      // fp32 screen: below lo surely closed, at or above hi surely open
+    float gate_mid, gate_hw;     // fp32 screen of the gate: fl(eps^2) and the half-width of the
+                                 // band around it inside which only the double comparison decides
+    float gate_keep;             // first pass keeps s - gate_mid >= gate_keep (normally -gate_hw)
     float clampv;                // output (FWD) or gradient (BWD) clamp; <= 0 off
     unsigned poll_limit;
 };
@@ -70,7 +77,7 @@ struct ScanSmem {
     static constexpr int NT = (KIND == KIND_BWD) ? 2 : 1;
     float4 tile[NT][TILE][32];
     float4 sE[W][32];
-    float4 sR[W][32];
+    float4 sR[kWindow + 1][32];
     float sCoef[64][6];
     unsigned long long epoch;
     int err;
@@ -78,26 +85,59 @@ struct ScanSmem {
 };
 
 __device__ __forceinline__ uint32_t smem_addr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void cp_async16(void *dst, const void *src)
+// Asynchronous global -> shared copies; the destination is a shared-space address plus a
+// compile-time byte offset, so that an unrolled loop needs no address arithmetic for it.
+template <int OFF>
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src)
 {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"(smem_addr(dst)), "l"(src) : "memory");
+    asm volatile("cp.async.cg.shared.global [%0+%2], [%1], 16;" :: "r"(dst), "l"(src), "n"(OFF) : "memory");
 }
-__device__ __forceinline__ void cp_async8(void *dst, const void *src)
+template <int OFF>
+__device__ __forceinline__ void cp_async8(uint32_t dst, const void *src)
 {
-    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" :: "r"(smem_addr(dst)), "l"(src) : "memory");
+    asm volatile("cp.async.ca.shared.global [%0+%2], [%1], 8;" :: "r"(dst), "l"(src), "n"(OFF) : "memory");
 }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
-
-// Copy (asynchronously) or zero one row piece of this lane: two adjacent complex64.
-template <bool VEC>
-__device__ __forceinline__ void fetch_piece(float4 *dst, const float2 *src, bool vA, bool vB)
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+// Wait until at most n of this thread's most recent copy groups are still in flight (n <= 4).
+__device__ __forceinline__ void cp_async_wait_pending(int n)
 {
+    switch (n) {
+    case 0: asm volatile("cp.async.wait_group 0;" ::: "memory"); break;
+    case 1: asm volatile("cp.async.wait_group 1;" ::: "memory"); break;
+    case 2: asm volatile("cp.async.wait_group 2;" ::: "memory"); break;
+    case 3: asm volatile("cp.async.wait_group 3;" ::: "memory"); break;
+    default: asm volatile("cp.async.wait_group 4;" ::: "memory"); break;
+    }
+}
+
+// Copy (asynchronously) or zero one row piece of this lane: two adjacent complex64 at byte
+// offset OFF from the thread's first piece (`dst` generic, `dst_s` the same in shared space).
+template <bool VEC, int OFF>
+__device__ __forceinline__ void fetch_piece(float4 *dst, uint32_t dst_s, const char *src, bool vA, bool vB)
+{
+    float4 *d4 = reinterpret_cast<float4 *>(reinterpret_cast<char *>(dst) + OFF);
     if (VEC) {
-        if (vA) cp_async16(dst, src); else *dst = zero4();
+        if (vA) cp_async16<OFF>(dst_s, src); else *d4 = zero4();
     } else {
-        float2 *d = reinterpret_cast<float2 *>(dst);
-        if (vA) cp_async8(d, src); else d[0] = make_float2(0.f, 0.f);
-        if (vB) cp_async8(d + 1, src + 1); else d[1] = make_float2(0.f, 0.f);
+        float2 *d = reinterpret_cast<float2 *>(d4);
+        if (vA) cp_async8<OFF>(dst_s, src); else d[0] = make_float2(0.f, 0.f);
+        if (vB) cp_async8<OFF + 8>(dst_s, src + 8); else d[1] = make_float2(0.f, 0.f);
+    }
+}
+
+// Unrolled helper: issue the T copies of one thread (rows i = 0..T-1, `step` bytes apart in
+// global memory, 512 bytes apart in shared memory), committing one copy group per GR rows
+// (GR = 0: the caller commits).  valid(i) says whether row i exists.
+template <bool VEC, int T, int GR, int I = 0, typename F>
+__device__ __forceinline__ void fetch_rows(float4 *dst, uint32_t dst_s, const char *src, long long step,
+                                           bool vA, bool vB, F valid)
+{
+    if constexpr (I < T) {
+        const bool row = valid(I);
+        fetch_piece<VEC, I * 512>(dst, dst_s, src, row && vA, row && vB);
+        if constexpr (GR > 0 && (I + 1) % GR == 0) cp_async_commit();
+        fetch_rows<VEC, T, GR, I + 1>(dst, dst_s, src + step, step, vA, vB, valid);
     }
 }
 
@@ -107,7 +147,7 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
 {
     constexpr bool REV = (KIND == KIND_BWD);
     constexpr int TILE = T * W;
-    constexpr int M = W - 1;
+    constexpr int M = kWindow;
     const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
     const int G = prm.G, C = prm.C, K = prm.K;
     const long long L = prm.L;
@@ -121,50 +161,47 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
     }
     // logical step s <-> physical row t: forward t = s, reverse t = L-1-s
     const long long t_first = REV ? (L - 1 - s0) : s0;
-    const long long rowstep = REV ? -(long long)C : (long long)C;  // in complex elements
+    const long long rowbytes = (REV ? -(long long)C : (long long)C) * 8;
     const long long e0 = ((long long)b * L + t_first) * C + c0;    // only used when nvalid > 0
     float4 *const xs = &sm.tile[0][w * T][lane];                   // this thread's pieces, 32 float4 apart
 
     // ---- 0. asynchronous copies into shared memory -----------------------------------------
-    {
-        const float2 *r = reinterpret_cast<const float2 *>(prm.in) + e0;
-#pragma unroll
-        for (int i = 0; i < T; ++i) {
-            const bool row = FULL || i < nvalid;
-            fetch_piece<VEC>(xs + i * 32, r, row && vA, row && vB);
-            r += rowstep;
-        }
-    }
+    // The rows go out as NG copy groups of GR rows each, so that phase 1 can start on the first
+    // rows while the later ones are still in flight.  The backward's second tile (needed in
+    // phase 3 only) is one more group behind them.
+    constexpr int GR = T < 4 ? T : 4, NG = T / GR;
+    static_assert(T % GR == 0 && NG <= 4, "copy groups");
+    fetch_rows<VEC, T, GR>(xs, smem_addr(xs), reinterpret_cast<const char *>(prm.in) + e0 * 8, rowbytes, vA, vB,
+                           [&](int i) { return FULL || i < nvalid; });
     if constexpr (KIND == KIND_BWD) {
         float4 *const qs = &sm.tile[1][w * T][lane];
         const bool have = prm.aux != nullptr;
-        const float2 *r = reinterpret_cast<const float2 *>(prm.aux) + e0 - C;   // row t-1
-#pragma unroll
-        for (int i = 0; i < T; ++i) {
-            const bool row = have && (FULL || i < nvalid) && (t_first - i >= 1);
-            fetch_piece<VEC>(qs + i * 32, r, row && vA, row && vB);
-            r += rowstep;
-        }
+        fetch_rows<VEC, T, 0>(qs, smem_addr(qs), reinterpret_cast<const char *>(prm.aux) + (e0 - C) * 8, rowbytes,
+                              vA, vB, [&](int i) { return have && (FULL || i < nvalid) && (t_first - i >= 1); });
+        cp_async_commit();
     }
 
     // ---- per-channel coefficients, in double, rounded once --------------------------------
-    if (tid < 64) {
-        const int ch = g * 64 + tid;
-        float cf[6] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    // Three independent tasks per channel, one thread each: a^n = gamma^n (cos n theta, sin n theta)
+    // for n = 1, T, TILE.  n theta is exact in double (theta is a float, n a small integer).
+    for (int idx = tid; idx < 192; idx += W * 32) {
+        const int task = idx >> 6, cl = idx & 63, ch = g * 64 + cl;
+        float re = 0.f, im = 0.f;
         if (ch < C) {
+            const int n = task == 0 ? 1 : (task == 1 ? T : TILE);
             const double gm = (double)prm.gamma[ch], th = (double)prm.theta[ch];
+            double mag = 1.0, base = gm;
+            for (int m = n; m > 0; m >>= 1) {            // gamma^n by square-and-multiply
+                if (m & 1) mag *= base;
+                base *= base;
+            }
             double sn, cs;
-            sincos(th, &sn, &cs);
-            const double ar = gm * cs, ai = REV ? -(gm * sn) : gm * sn;
-            double tr, ti, wr, wi;
-            cpow_int<T>(ar, ai, tr, ti);
-            cpow_int<W>(tr, ti, wr, wi);
-            cf[0] = (float)ar; cf[1] = (float)ai;
-            cf[2] = (float)tr; cf[3] = (float)ti;
-            cf[4] = (float)wr; cf[5] = (float)wi;
+            sincos(th * (double)n, &sn, &cs);
+            re = (float)(mag * cs);
+            im = (float)(REV ? -(mag * sn) : mag * sn);
         }
-#pragma unroll
-        for (int i = 0; i < 6; ++i) sm.sCoef[tid][i] = cf[i];
+        sm.sCoef[cl][2 * task] = re;
+        sm.sCoef[cl][2 * task + 1] = im;
     }
     unsigned long long epoch0 = 0;
     unsigned arrived = 0;
@@ -185,9 +222,20 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
         aT = make_float4(u0.z, u0.w, u2.x, u2.y);
     }
     const unsigned long long epoch = sm.epoch;
-    cp_async_wait_all();                                  // this thread's pieces have landed
+
+    // Window of carry records this tile needs (see the header comment), and a first,
+    // non-blocking reading of the record this warp is responsible for: it is usually there
+    // already, and its latency then hides behind phase 1.
+    const long long chain = (long long)b * G + g;
+    const int cpt = k > 0 ? M * ((k - 1) / M) : 0;       // last checkpoint before this tile
+    const int nrec = k - cpt;                            // aggregates in the window, 0..M
+    const uint4 *early_ptr = nullptr;
+    if (w < nrec) early_ptr = prm.agg + (chain * K + (k - 1 - w)) * 64;
+    else if (w == M && cpt > 0) early_ptr = prm.pre + (chain * prm.KP + cpt / M) * 64;
+    uint4 er0 = make_uint4(0u, 0u, 0u, 0u), er1 = er0;
 
     if constexpr (KIND == KIND_BWD) {
+        cp_async_wait_all();
         // the step at t = 0 multiplies the call's initial state; lam_{L-1} = G_{L-1} + grad_state_out
         if (nvalid > 0 && t_first - (nvalid - 1) == 0 && prm.aux != nullptr && prm.state_in != nullptr) {
             const float2 *r = prm.state_in + (long long)b * C + c0;
@@ -210,48 +258,75 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
     if constexpr (KIND == KIND_FWD) {
         // |p| >= eps decided as re^2 + im^2 >= eps^2 in double: both squares are exact there
         // and the sum rounds once, so the decision is reproducible bit for bit.  The fp32 sum
-        // of squares is within 2^-22 of the exact one, so it settles every case outside a
-        // 2^-21 band around the threshold; a row with a lane in the band takes the double path.
-        const float lo = prm.gate_lo, hi = prm.gate_hi;
+        // of squares s is within 2^-22 (relative) of the exact one, so d = s - mid, mid =
+        // fl(eps^2), settles every case with |d| > hw = 2^-20 mid.  The first pass keeps
+        // everything with d >= keep = -hw and remembers the smallest |d| it saw; if any lane of
+        // the warp saw one inside the band, the warp redoes its rows with the double comparison
+        // (shared memory still holds the original of every element the first pass kept).
+        const float mid = prm.gate_mid, hw = prm.gate_hw, keep = prm.gate_keep;
         const bool want_mask = prm.mask != nullptr;
-        uint32_t *mrow = prm.mask + ((long long)b * L + s0) * prm.MW + g * 2;
+        uint32_t *const mrow0 = prm.mask + ((long long)b * L + s0) * prm.MW + g * 2;
         const bool second_word = g * 2 + 1 < prm.MW;
+        auto pass = [&](auto exact_tag, auto mask_tag) -> float {
+            constexpr bool EXACT = decltype(exact_tag)::value, MASK = decltype(mask_tag)::value;
+            float nearest = INFINITY;
+            uint32_t *mrow = mrow0;
+            e = zero4();
 #pragma unroll
-        for (int i = 0; i < T; ++i) {
-            float4 v = xs[i * 32];
-            const float sA = fmaf(v.x, v.x, v.y * v.y), sB = fmaf(v.z, v.z, v.w * v.w);
-            bool oA = sA >= hi, oB = sB >= hi;
-            const bool band = (!oA && sA >= lo) || (!oB && sB >= lo);
-            if (__any_sync(0xffffffffu, band)) {
-                oA = ((double)v.x * (double)v.x + (double)v.y * (double)v.y >= prm.eps2);
-                oB = ((double)v.z * (double)v.z + (double)v.w * (double)v.w >= prm.eps2);
-            }
-            if (!FULL) { oA = oA && vA; oB = oB && vB; }
-            if (!(oA && oB)) {
-                if (!oA) { v.x = 0.f; v.y = 0.f; }
-                if (!oB) { v.z = 0.f; v.w = 0.f; }
-                xs[i * 32] = v;
-            }
-            if (want_mask) {
-                // lanes 0..15 hold channels 0..31 of the group (word 0), lanes 16..31 word 1
-                const unsigned bits = ((oA ? 1u : 0u) | (oB ? 2u : 0u)) << (2 * (lane & 15));
-                const unsigned w0 = __reduce_or_sync(0xffffffffu, lane < 16 ? bits : 0u);
-                const unsigned w1 = __reduce_or_sync(0xffffffffu, lane < 16 ? 0u : bits);
-                if (FULL || i < nvalid) {
-                    if (lane == 0) mrow[0] = w0;
-                    if (lane == 16 && second_word) mrow[1] = w1;
+            for (int i = 0; i < T; ++i) {
+                if (!EXACT && i % GR == 0) {
+                    cp_async_wait_pending(NG - 1 - i / GR);       // rows i .. i+GR-1 have landed
+                    if (i == 0 && early_ptr != nullptr) {
+                        er0 = ld_record(early_ptr + 2 * lane);
+                        er1 = ld_record(early_ptr + 2 * lane + 1);
+                    }
                 }
-                mrow += prm.MW;
+                float4 v = xs[i * 32];
+                bool oA, oB;
+                if (EXACT) {
+                    oA = ((double)v.x * (double)v.x + (double)v.y * (double)v.y >= prm.eps2);
+                    oB = ((double)v.z * (double)v.z + (double)v.w * (double)v.w >= prm.eps2);
+                } else {
+                    const float dA = fmaf(v.x, v.x, v.y * v.y) - mid, dB = fmaf(v.z, v.z, v.w * v.w) - mid;
+                    nearest = fminf(nearest, fminf(fabsf(dA), fabsf(dB)));
+                    oA = dA >= keep; oB = dB >= keep;
+                }
+                if (!FULL) { oA = oA && vA; oB = oB && vB; }
+                v.x = oA ? v.x : 0.f; v.y = oA ? v.y : 0.f;
+                v.z = oB ? v.z : 0.f; v.w = oB ? v.w : 0.f;
+                xs[i * 32] = v;                           // phase 3 reads the gated value
+                if (MASK) {
+                    // lanes 0..15 hold channels 0..31 of the group (word 0), lanes 16..31 word 1
+                    const unsigned bits = ((oA ? 1u : 0u) | (oB ? 2u : 0u)) << (2 * (lane & 15));
+                    const unsigned w0 = __reduce_or_sync(0xffffffffu, lane < 16 ? bits : 0u);
+                    const unsigned w1 = __reduce_or_sync(0xffffffffu, lane < 16 ? 0u : bits);
+                    if (FULL || i < nvalid) {
+                        if (lane == 0) mrow[0] = w0;
+                        if (lane == 16 && second_word) mrow[1] = w1;
+                    }
+                    mrow += prm.MW;
+                }
+                if (FULL || i < nvalid) e = cfma2(a, e, v);
             }
-            if (FULL || i < nvalid) e = cfma2(a, e, v);
+            return nearest;
+        };
+        using yes = std::true_type;
+        using no = std::false_type;
+        const float nearest = want_mask ? pass(no{}, yes{}) : pass(no{}, no{});
+        if (__any_sync(0xffffffffu, nearest <= hw)) {
+            if (want_mask) pass(yes{}, yes{}); else pass(yes{}, no{});
         }
     } else {
+        if (early_ptr != nullptr) {
+            er0 = ld_record(early_ptr + 2 * lane);
+            er1 = ld_record(early_ptr + 2 * lane + 1);
+        }
 #pragma unroll
         for (int i = 0; i < T; ++i)
             if (FULL || i < nvalid) e = cfma2(a, e, xs[i * 32]);
     }
     sm.sE[w][lane] = e;
-    if (tid == 0 && arrived == gridDim.x - 1) {
+    if (tid == 0 && arrived == gridDim.x * gridDim.y * gridDim.z - 1) {
         // every CTA of this launch has read the epoch: open the next one
         st_volatile_u32(&prm.ws->done, 0u);
         st_volatile_u64(&prm.ws->epoch, epoch0 + 1ull);
@@ -259,30 +334,32 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
     __syncthreads();                                                           // barrier 2
 
     // ---- 2. publish the aggregate, fetch the carry window ----------------------------------
-    const long long chain = (long long)b * G + g;
-    const int cpt = k > 0 ? M * ((k - 1) / M) : 0;       // last checkpoint before this tile
-    const int nrec = k - cpt;                            // aggregates in the window, 0..M
     if (w == 0 && k + 1 < K) {
         float4 E = sm.sE[0][lane];
 #pragma unroll
         for (int i = 1; i < W; ++i) E = cfma2(aT, E, sm.sE[i][lane]);
         publish_pair(prm.agg + (chain * K + k) * 64, lane, E, epoch, REC_AGGREGATE);
     }
-    {
+    // slot r < nrec of the window: aggregate of tile k-1-r; slot M: the carry-in the window starts from
+    for (int slot = w; slot <= M; slot += W) {
         float4 r = zero4();
         bool ok = true;
-        if (w < nrec) {
-            ok = poll_pair(prm.agg + (chain * K + (k - 1 - w)) * 64, lane, epoch, prm.poll_limit, r);
-        } else if (w == W - 1) {
+        const uint4 none = make_uint4(0u, 0u, 0u, 0u);
+        const bool mine = (slot == w);                   // the slot read ahead of phase 1
+        if (slot < nrec) {
+            ok = poll_pair(prm.agg + (chain * K + (k - 1 - slot)) * 64, lane, epoch, prm.poll_limit,
+                           mine ? er0 : none, mine ? er1 : none, r);
+        } else if (slot == M) {
             if (cpt > 0) {
-                ok = poll_pair(prm.pre + (chain * prm.KP + cpt / M) * 64, lane, epoch, prm.poll_limit, r);
+                ok = poll_pair(prm.pre + (chain * prm.KP + cpt / M) * 64, lane, epoch, prm.poll_limit,
+                               mine ? er0 : none, mine ? er1 : none, r);
             } else if (!REV && prm.state_in != nullptr) {
                 const float2 *s = prm.state_in + (long long)b * C + c0;
                 if (vA) { const float2 v = s[0]; r.x = v.x; r.y = v.y; }
                 if (vB) { const float2 v = s[1]; r.z = v.x; r.w = v.y; }
             }
         }
-        sm.sR[w][lane] = r;
+        sm.sR[slot][lane] = r;
         if (!ok) {
             sm.err = 1;
             atomicMax(&prm.ws->status, 1u);              // CAWN_ERR_CARRY_TIMEOUT
@@ -295,34 +372,31 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
     const bool checkpoint = (k > 0 && k % M == 0 && k + 1 < K);
     float4 qa = zero4();
     if (!failed) {
-        float4 P = sm.sR[W - 1][lane];
+        float4 P = sm.sR[M][lane];
         {
             const float4 *cp = reinterpret_cast<const float4 *>(&sm.sCoef[2 * lane][0]);
             const float4 u1 = cp[1], u2 = cp[2];
             const float4 AA = make_float4(u1.x, u1.y, u2.z, u2.w);
-#pragma unroll
-            for (int i = M - 1; i >= 0; --i)
-                if (i < nrec) P = cfma2(AA, P, sm.sR[i][lane]);
+#pragma unroll 1
+            for (int i = nrec - 1; i >= 0; --i) P = cfma2(AA, P, sm.sR[i][lane]);
         }
         if (checkpoint && w == 0)
             publish_pair(prm.pre + (chain * prm.KP + k / M) * 64, lane, P, epoch, REC_PREFIX);
-#pragma unroll
-        for (int i = 0; i < W - 1; ++i)
-            if (i < w) P = cfma2(aT, P, sm.sE[i][lane]);
+#pragma unroll 1
+        for (int i = 0; i < w; ++i) P = cfma2(aT, P, sm.sE[i][lane]);
 
-        float2 *r = reinterpret_cast<float2 *>(prm.out) + e0;
+        char *r = reinterpret_cast<char *>(prm.out) + e0 * 8;
         const float cl = prm.clampv;
-        const bool clamped = cl > 0.f;
-#pragma unroll
-        for (int i = 0; i < T; ++i) {
+        auto step_row = [&](int i, bool clamped) {
             if (FULL || i < nvalid) {
                 P = cfma2(a, P, xs[i * 32]);
                 const float4 o = clamped ? clamp4(P, cl) : P;
                 if (VEC) {
                     if (vA) __stcs(reinterpret_cast<float4 *>(r), o);
                 } else {
-                    if (vA) __stcs(r, make_float2(o.x, o.y));
-                    if (vB) __stcs(r + 1, make_float2(o.z, o.w));
+                    float2 *r2 = reinterpret_cast<float2 *>(r);
+                    if (vA) __stcs(r2, make_float2(o.x, o.y));
+                    if (vB) __stcs(r2 + 1, make_float2(o.z, o.w));
                 }
                 if constexpr (KIND == KIND_BWD) {
                     // conj(lam) * P_{t-1}
@@ -333,7 +407,14 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
                     qa.w = fmaf(P.z, q.w, fmaf(-P.w, q.z, qa.w));
                 }
             }
-            r += rowstep;
+            r += rowbytes;
+        };
+        if (cl > 0.f) {
+#pragma unroll
+            for (int i = 0; i < T; ++i) step_row(i, true);
+        } else {
+#pragma unroll
+            for (int i = 0; i < T; ++i) step_row(i, false);
         }
         // the thread that owns the last step writes the carried state (never clamped)
         if (prm.state_out != nullptr && nvalid > 0 && s0 + nvalid == L) {
@@ -372,10 +453,10 @@ __global__ void __launch_bounds__(W * 32, MINB) cawn_scan_kernel(const ScanParam
     extern __shared__ __align__(128) unsigned char smem_raw[];
     ScanSmem<T, W, KIND> &sm = *reinterpret_cast<ScanSmem<T, W, KIND> *>(smem_raw);
 
-    const int g = blockIdx.x % prm.G;
-    const int bk = blockIdx.x / prm.G;
-    const int b = bk % prm.B;
-    const int k = bk / prm.B;                         // tile index along (logical) time
+    // grid = (G, B, K): blocks are dispatched x fastest, so a tile's predecessors along time
+    // (smaller k) always have smaller linear block indices
+    const int g = blockIdx.x, b = blockIdx.y;
+    const int k = blockIdx.z;                         // tile index along (logical) time
     const bool full = ((long long)(k + 1) * TILE <= prm.L) && (g * 64 + 64 <= prm.C);
     if (full) scan_tile<T, W, KIND, VEC, true>(prm, sm, g, b, k);
     else      scan_tile<T, W, KIND, VEC, false>(prm, sm, g, b, k);
