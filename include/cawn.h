@@ -53,6 +53,8 @@ typedef enum cawn_status {
     CAWN_ERR_UNSUPPORTED          = -4,  /* valid request this build has no kernel for           */
     CAWN_ERR_WORKSPACE_TOO_SMALL  = -5,
     CAWN_ERR_CUDA                 = -6,  /* a CUDA runtime call failed (launch, copy)            */
+    CAWN_ERR_STATIC_TOO_LARGE     = -7,  /* cawn_phase_accumulate_fwd_static: the call needs more
+                                            scratch than the library's built-in array holds      */
     CAWN_ERR_CARRY_TIMEOUT        = 1    /* device: an inter-tile carry wait hit its bound;
                                             outputs of that call are incomplete                  */
 } cawn_status;
@@ -197,6 +199,47 @@ CAWN_API int cawn_phase_accumulate_fwd_host(const cawn_params *params,
                                             uint32_t *gate_mask_host,
                                             void *device_scratch, size_t device_scratch_bytes,
                                             void *cuda_stream);
+
+/*
+ * Forward phase accumulation for callers that cannot allocate device memory.  (The paper has
+ * no counterpart: this is a packaging variant of cawn_phase_accumulate_fwd, same arithmetic.)
+ *
+ * Who needs it: code that runs where a cudaMalloc is not an option -- a plugin inside a serving
+ * process whose device memory has all been handed to one framework-owned pool, a callback that
+ * must not block on the allocator or synchronise the device, or a component that is given
+ * input and output buffers and nothing else.  Such a caller cannot provide the carry workspace
+ * the ordinary entry point asks for, so this one uses a scratch array compiled into the library
+ * instead: a file-scope __device__ array of CAWN_STATIC_SCRATCH_BYTES (4 MiB), which every GPU
+ * that loads the library holds until the process exits.
+ *
+ * Same operation and arguments as the Cartesian, static-retention cawn_phase_accumulate_fwd
+ * (conv_k == 0, no CAWN_FLAG_RETENTION_DYNAMIC), without the workspace pair.
+ * device_status: device pointer to one uint32 or NULL.  When given, the device-side status of
+ *               this call (0 or CAWN_ERR_CARRY_TIMEOUT) is copied there on the stream after the
+ *               kernel; there is no separate poll call for the built-in scratch.
+ *
+ * Limits and rules.
+ *  - The call is rejected with CAWN_ERR_STATIC_TOO_LARGE, before anything is launched, when
+ *    cawn_workspace_bytes(params, CAWN_OP_FWD) exceeds CAWN_STATIC_SCRATCH_BYTES.  The need is
+ *    256 + B * ceil(C/64) * (K + K/7 + 1) * 1024 bytes with K = ceil(L/128) tiles: 1.9 MB for
+ *    B=8, L=2048, C=768; about 4,000 (batch x 64-channel group x tile) units in all.
+ *  - It calls no cudaMalloc/cudaFree and no allocating library routine.
+ *  - The first call on each device looks up the array's device address (one
+ *    cudaGetSymbolAddress with that device current) and remembers it; make that first call
+ *    outside any stream capture.
+ *  - All calls on a device share the one array, and it keeps what the last call left in it.
+ *    The kernel's epoch tags make stale records harmless and the status word is cleared at the
+ *    start of every call, but two calls that overlap on the GPU (different streams, or
+ *    different host threads) race on it: serialise them.
+ */
+#define CAWN_STATIC_SCRATCH_BYTES (4u << 20)
+CAWN_API int cawn_phase_accumulate_fwd_static(const cawn_params *params,
+                                              const void *input,
+                                              const float *gamma, const float *theta,
+                                              const void *state_in,
+                                              void *y, void *state_out, uint32_t *gate_mask,
+                                              uint32_t *device_status,
+                                              void *cuda_stream);
 
 #ifdef __cplusplus
 }

@@ -20,6 +20,8 @@ CAWN_ERR_MISALIGNED = -3
 CAWN_ERR_UNSUPPORTED = -4
 CAWN_ERR_WORKSPACE_TOO_SMALL = -5
 CAWN_ERR_CUDA = -6
+CAWN_ERR_STATIC_TOO_LARGE = -7
+CAWN_STATIC_SCRATCH_BYTES = 4 << 20
 CAWN_ERR_CARRY_TIMEOUT = 1
 
 CAWN_FLAG_PRELUDE_CLAMP_SILU = 1
@@ -31,7 +33,7 @@ CAWN_SAVED_STATES, CAWN_SAVED_PUSHES = 0, 1
 EXPORTS = (
     "cawn_status_string", "cawn_workspace_bytes", "cawn_workspace_init",
     "cawn_phase_accumulate_fwd", "cawn_phase_accumulate_bwd", "cawn_state_carry",
-    "cawn_poll_status", "cawn_phase_accumulate_fwd_host",
+    "cawn_poll_status", "cawn_phase_accumulate_fwd_host", "cawn_phase_accumulate_fwd_static",
 )
 
 
@@ -80,6 +82,7 @@ def lib():
         L.cawn_state_carry.argtypes = [pp, vp, vp, ctypes.c_int64, fp, fp, vp, vp]
         L.cawn_poll_status.argtypes = [vp, vp]
         L.cawn_phase_accumulate_fwd_host.argtypes = [pp, vp, fp, fp, vp, vp, vp, vp, vp, sz, vp]
+        L.cawn_phase_accumulate_fwd_static.argtypes = [pp, vp, fp, fp, vp, vp, vp, vp, vp, vp]
         for name in EXPORTS:
             if name != "cawn_status_string":
                 getattr(L, name).restype = ctypes.c_int
@@ -176,3 +179,13 @@ def cawn_phase_accumulate_fwd_host(params, p_host, gamma_host, theta_host, y_hos
         _dp(y_host), _dp(state_out_host), _dp(gate_mask_host), _dp(device_scratch),
         device_scratch.numel() * device_scratch.element_size(), _stream(stream)),
         "cawn_phase_accumulate_fwd_host")
+
+
+def cawn_phase_accumulate_fwd_static(params, input, gamma, theta, y, state_in=None, state_out=None,
+                                     gate_mask=None, device_status=None, stream=None):
+    """Forward scan on the library's built-in scratch array: for callers that hold input and
+    output buffers but cannot allocate a workspace.  One call at a time per device."""
+    _check(lib().cawn_phase_accumulate_fwd_static(
+        ctypes.byref(params), _dp(input), _dp(gamma), _dp(theta), _dp(state_in), _dp(y),
+        _dp(state_out), _dp(gate_mask), _dp(device_status), _stream(stream)),
+        "cawn_phase_accumulate_fwd_static")

@@ -155,6 +155,27 @@ HostStage host_stage(const cawn_params *p)
     return h;
 }
 
+// Built-in scratch of cawn_phase_accumulate_fwd_static: lives in every GPU that loads the
+// library.  In host code this name is only a handle; the device address comes from
+// cudaGetSymbolAddress, looked up once per device.
+static __device__ __align__(256) unsigned char g_static_scratch[CAWN_STATIC_SCRATCH_BYTES];
+
+cudaError_t static_scratch_address(void **out)
+{
+    static void *address[64] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev >= 0 && dev < 64 && address[dev] != nullptr) { *out = address[dev]; return cudaSuccess; }
+    void *p = nullptr;
+    e = cudaGetSymbolAddress(&p, g_static_scratch);
+    if (e != cudaSuccess) return e;
+    if (p == nullptr) return cudaErrorInvalidSymbol;
+    if (dev >= 0 && dev < 64) address[dev] = p;
+    *out = p;
+    return cudaSuccess;
+}
+
 }  // namespace
 
 extern "C" {
@@ -169,6 +190,7 @@ const char *cawn_status_string(int status)
     case CAWN_ERR_UNSUPPORTED: return "request not supported by this build";
     case CAWN_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
     case CAWN_ERR_CUDA: return "CUDA runtime error";
+    case CAWN_ERR_STATIC_TOO_LARGE: return "call needs more scratch than the built-in array holds";
     case CAWN_ERR_CARRY_TIMEOUT: return "device: inter-tile carry wait ran out";
     default: return "unknown status";
     }
@@ -442,6 +464,32 @@ int cawn_phase_accumulate_fwd_host(const cawn_params *params, const void *p_host
     if (gate_mask_host && mask_bytes)
         ok &= cudaMemcpyAsync(gate_mask_host, d + h.off_mask, mask_bytes, cudaMemcpyDeviceToHost, st) == cudaSuccess;
     return ok ? CAWN_OK : CAWN_ERR_CUDA;
+}
+
+int cawn_phase_accumulate_fwd_static(const cawn_params *params, const void *input,
+                                     const float *gamma, const float *theta, const void *state_in,
+                                     void *y, void *state_out, uint32_t *gate_mask,
+                                     uint32_t *device_status, void *cuda_stream)
+{
+    size_t need = 0;
+    int rc = cawn_workspace_bytes(params, CAWN_OP_FWD, &need);
+    if (rc != CAWN_OK) return rc;
+    if (need > (size_t)CAWN_STATIC_SCRATCH_BYTES) return CAWN_ERR_STATIC_TOO_LARGE;
+    if (!aligned(device_status, 4)) return CAWN_ERR_MISALIGNED;
+    void *scratch = nullptr;
+    if (static_scratch_address(&scratch) != cudaSuccess) return CAWN_ERR_CUDA;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    WsHeader *ws = reinterpret_cast<WsHeader *>(scratch);
+    // the array keeps the previous call's contents: only the sticky status has to start at zero
+    if (cudaMemsetAsync(&ws->status, 0, sizeof(unsigned), st) != cudaSuccess) return CAWN_ERR_CUDA;
+    rc = cawn_phase_accumulate_fwd(params, input, gamma, theta, nullptr, nullptr, nullptr, nullptr,
+                                   state_in, y, state_out, gate_mask, scratch,
+                                   (size_t)CAWN_STATIC_SCRATCH_BYTES, st);
+    if (rc != CAWN_OK) return rc;
+    if (device_status != nullptr &&
+        cudaMemcpyAsync(device_status, &ws->status, sizeof(unsigned), cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+        return CAWN_ERR_CUDA;
+    return CAWN_OK;
 }
 
 }  // extern "C"
