@@ -129,6 +129,11 @@ inline cudaError_t launch_fwd(TileShape ts, const ScanParams &sp, cudaStream_t s
     if (ts.T == 16) return launch_scan<16, 8, KIND_FWD, 3>(sp, st);
     return launch_scan<4, 4, KIND_FWD, 8>(sp, st);
 }
+inline cudaError_t launch_fused(TileShape ts, const ScanParams &sp, cudaStream_t st)
+{
+    if (ts.T == 16) return launch_scan<16, 8, KIND_FUSED, 3>(sp, st);
+    return launch_scan<4, 4, KIND_FUSED, 8>(sp, st);
+}
 inline cudaError_t launch_bwd(TileShape ts, const ScanParams &sp, cudaStream_t st)
 {
     if (ts.T == 8) return launch_scan<8, 8, KIND_BWD, 3>(sp, st);
@@ -250,9 +255,17 @@ int cawn_phase_accumulate_fwd(const cawn_params *params, const void *input,
 {
     int rc = check_params(params);
     if (rc != CAWN_OK) return rc;
-    (void)conv_w; (void)conv_bias; (void)gamma_logit; (void)freq_bias;
-    if (params->conv_k != 0 || (params->flags & CAWN_FLAG_RETENTION_DYNAMIC))
-        return CAWN_ERR_UNSUPPORTED;
+    (void)gamma_logit; (void)freq_bias;
+    if (params->flags & CAWN_FLAG_RETENTION_DYNAMIC) return CAWN_ERR_UNSUPPORTED;
+    const bool fused = params->conv_k != 0;
+    if (fused) {
+        if (params->conv_k > 4) return CAWN_ERR_UNSUPPORTED;
+        if (conv_w == nullptr) return CAWN_ERR_NULL_POINTER;
+        // with clamp + SiLU the magnitude is at least 0.43: thresholds below that leave every gate
+        // open, which is what the kernel assumes; higher ones are not provided for
+        if ((params->flags & CAWN_FLAG_PRELUDE_CLAMP_SILU) && params->gate_eps > 0.4f) return CAWN_ERR_UNSUPPORTED;
+        if (!aligned(conv_w, 4) || !aligned(conv_bias, 4)) return CAWN_ERR_MISALIGNED;
+    }
     if (gamma == nullptr || theta == nullptr || workspace == nullptr) return CAWN_ERR_NULL_POINTER;
     if (params->L > 0 && (input == nullptr || y == nullptr)) return CAWN_ERR_NULL_POINTER;
     if (!aligned(input, 16) || !aligned(y, 16) || !aligned(workspace, 16) ||
@@ -265,9 +278,9 @@ int cawn_phase_accumulate_fwd(const cawn_params *params, const void *input,
     if (workspace_bytes < sizeof(WsHeader) + g.rec_bytes) return CAWN_ERR_WORKSPACE_TOO_SMALL;
     cudaStream_t st = (cudaStream_t)cuda_stream;
 
-    if (params->L == 0) {               // nothing to scan: the state passes through
+    if (params->L == 0) {               // nothing to scan: the state (and conv history) passes through
         if (state_out != nullptr && state_out != state_in) {
-            const size_t nb = (size_t)params->B * g.C * sizeof(float2);
+            const size_t nb = fused ? state_blob_bytes(params) : (size_t)params->B * g.C * sizeof(float2);
             cudaError_t e = state_in ? cudaMemcpyAsync(state_out, state_in, nb, cudaMemcpyDeviceToDevice, st)
                                      : cudaMemsetAsync(state_out, 0, nb, st);
             if (e != cudaSuccess) return CAWN_ERR_CUDA;
@@ -288,6 +301,20 @@ int cawn_phase_accumulate_fwd(const cawn_params *params, const void *input,
     set_gate(sp, params->gate_eps);
     sp.clampv = params->clamp_abs > 0.f ? params->clamp_abs : 0.f;
     sp.poll_limit = kPollLimit;
+    if (fused) {
+        // state blob: P [B,C] complex64, then (16-byte aligned) the conv history [B,conv_k-1,C]
+        const size_t tail_off = round_up((size_t)params->B * g.C * sizeof(float2), 16);
+        sp.conv_w = conv_w; sp.conv_bias = conv_bias;
+        sp.conv_k = params->conv_k;
+        sp.clamp_silu = (params->flags & CAWN_FLAG_PRELUDE_CLAMP_SILU) ? 1 : 0;
+        sp.gate_tau = params->gate_tau;
+        if (params->conv_k > 1) {
+            sp.tail_in = state_in ? reinterpret_cast<const float *>(reinterpret_cast<const char *>(state_in) + tail_off) : nullptr;
+            sp.tail_out = state_out ? reinterpret_cast<float *>(reinterpret_cast<char *>(state_out) + tail_off) : nullptr;
+        }
+        if (launch_fused(ts, sp, st) != cudaSuccess) return CAWN_ERR_CUDA;
+        return CAWN_OK;
+    }
     if (launch_fwd(ts, sp, st) != cudaSuccess) return CAWN_ERR_CUDA;
     return CAWN_OK;
 }

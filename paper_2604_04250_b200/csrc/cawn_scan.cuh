@@ -41,13 +41,17 @@
 
 namespace cawn {
 
-enum : int { KIND_FWD = 0, KIND_BWD = 2 };
+enum : int { KIND_FWD = 0, KIND_FUSED = 1, KIND_BWD = 2 };
+
+// Rows of hidden-state history in front of a tile that the fused conv prelude may read.
+constexpr int kHalo = 3;
 
 // Carry window: every kWindow-th tile of a chain is a checkpoint.
 constexpr int kWindow = 7;
 
 struct ScanParams {
     const void *in;              // FWD: pushes p;  BWD: grad_y              [B,L,C] complex64
+                                 // FUSED: hidden states h                   [B,L,C] float
     void *out;                   // FWD: y;         BWD: grad_p
     const void *aux;             // BWD: saved unclamped states P (NULL: no parameter sums)
     const float *gamma, *theta;  // [C]
@@ -67,6 +71,14 @@ struct ScanParams {
     float gate_keep;             // first pass keeps s - gate_mid >= gate_keep (normally -gate_hw)
     float clampv;                // output (FWD) or gradient (BWD) clamp; <= 0 off
     unsigned poll_limit;
+    // fused conv prelude (KIND_FUSED)
+    const float *conv_w;         // [C][conv_k]
+    const float *conv_bias;      // [C] or NULL
+    const float *tail_in;        // [B][conv_k-1][C] carried hidden rows or NULL (zeros)
+    float *tail_out;             // [B][conv_k-1][C] or NULL
+    int conv_k;                  // 1..4
+    int clamp_silu;              // clamp the conv output to +-50, then SiLU
+    float gate_tau;              // gate: conv output >= gate_tau (fp32 fmaf chain, tap order)
 };
 
 // Shared memory of one CTA: the tile (two tiles in the backward: grad_y and P_{t-1}), then the
@@ -96,6 +108,10 @@ template <int OFF>
 __device__ __forceinline__ void cp_async8(uint32_t dst, const void *src)
 {
     asm volatile("cp.async.ca.shared.global [%0+%2], [%1], 8;" :: "r"(dst), "l"(src), "n"(OFF) : "memory");
+}
+__device__ __forceinline__ void cp_async4(uint32_t dst, const void *src)
+{
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" :: "r"(dst), "l"(src) : "memory");
 }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
@@ -171,8 +187,47 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
     // phase 3 only) is one more group behind them.
     constexpr int GR = T < 4 ? T : 4, NG = T / GR;
     static_assert(T % GR == 0 && NG <= 4, "copy groups");
-    fetch_rows<VEC, T, GR>(xs, smem_addr(xs), reinterpret_cast<const char *>(prm.in) + e0 * 8, rowbytes, vA, vB,
-                           [&](int i) { return FULL || i < nvalid; });
+    // Fused path: the hidden rows (floats) are staged in the upper part of the tile, behind
+    // kHalo rows of history; phase 1 takes them into registers before the pushes overwrite them.
+    float *const hs = reinterpret_cast<float *>(&sm.tile[0][0][0]) + (TILE * 128 - (TILE + kHalo) * 64);
+    if constexpr (KIND == KIND_FUSED) {
+        const float *hin = reinterpret_cast<const float *>(prm.in);
+        float *mine = hs + (kHalo + w * T) * 64 + 2 * lane;
+        const float *r = hin + e0;
+#pragma unroll
+        for (int i = 0; i < T; ++i) {
+            const bool row = FULL || i < nvalid;
+            float *d = mine + i * 64;
+            if (VEC) {
+                if (row && vA) cp_async8<0>(smem_addr(d), r); else *reinterpret_cast<float2 *>(d) = make_float2(0.f, 0.f);
+            } else {
+                if (row && vA) cp_async4(smem_addr(d), r); else d[0] = 0.f;
+                if (row && vB) cp_async4(smem_addr(d + 1), r + 1); else d[1] = 0.f;
+            }
+            r += C;
+        }
+        // history rows in front of the tile: earlier rows of h, or the carried tail before t = 0
+        const int Kh = prm.conv_k - 1;
+        if (w == 0) {
+            const long long t0 = (long long)k * TILE;
+#pragma unroll
+            for (int j = 0; j < kHalo; ++j) {
+                const long long t = t0 - kHalo + j;
+                float *d = hs + j * 64 + 2 * lane;
+                const float *src = nullptr;
+                if (j >= kHalo - Kh) {
+                    if (t >= 0) src = hin + ((long long)b * L + t) * C + c0;
+                    else if (prm.tail_in != nullptr) src = prm.tail_in + ((long long)b * Kh + (Kh + t)) * C + c0;
+                }
+                if (src != nullptr && vA) cp_async4(smem_addr(d), src); else d[0] = 0.f;
+                if (src != nullptr && vB) cp_async4(smem_addr(d + 1), src + 1); else d[1] = 0.f;
+            }
+        }
+        cp_async_commit();
+    } else {
+        fetch_rows<VEC, T, GR>(xs, smem_addr(xs), reinterpret_cast<const char *>(prm.in) + e0 * 8, rowbytes, vA, vB,
+                               [&](int i) { return FULL || i < nvalid; });
+    }
     if constexpr (KIND == KIND_BWD) {
         float4 *const qs = &sm.tile[1][w * T][lane];
         const bool have = prm.aux != nullptr;
@@ -212,6 +267,7 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
         // counted only once the epoch has been read (the increment depends on its value)
         arrived = atomicAdd(&prm.ws->done, 1u + (unsigned)(epoch0 >> 63));
     }
+    if constexpr (KIND == KIND_FUSED) cp_async_wait_all();   // rows are read across threads below
     __syncthreads();                                                           // barrier 1
     float4 a, aT;
     {
@@ -233,6 +289,14 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
     if (w < nrec) early_ptr = prm.agg + (chain * K + (k - 1 - w)) * 64;
     else if (w == M && cpt > 0) early_ptr = prm.pre + (chain * prm.KP + cpt / M) * 64;
     uint4 er0 = make_uint4(0u, 0u, 0u, 0u), er1 = er0;
+    // The call's initial state is read before this tile publishes anything, so that state_out
+    // may alias state_in: whoever writes state_out has waited for every tile's aggregate.
+    float4 sinit = zero4();
+    if (!REV && cpt == 0 && w == M % W && prm.state_in != nullptr) {
+        const float2 *sp = prm.state_in + (long long)b * C + c0;
+        if (vA) { const float2 v = sp[0]; sinit.x = v.x; sinit.y = v.y; }
+        if (vB) { const float2 v = sp[1]; sinit.z = v.x; sinit.w = v.y; }
+    }
 
     if constexpr (KIND == KIND_BWD) {
         cp_async_wait_all();
@@ -255,7 +319,83 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
 
     // ---- 1. gate + local reduction from a zero start ---------------------------------------
     float4 e = zero4();
-    if constexpr (KIND == KIND_FWD) {
+    if constexpr (KIND == KIND_FUSED) {
+        // Temporal Syntax Cache prelude: causal depthwise conv over time (taps right-aligned on
+        // the current token, fmaf chain in tap order from the bias), optional clamp + SiLU,
+        // magnitude sigmoid(x), phase pi*tanh(x), gate on the conv output, push m (cos, sin).
+        float2 hv[T + kHalo];
+#pragma unroll
+        for (int r = 0; r < T + kHalo; ++r)
+            hv[r] = *reinterpret_cast<const float2 *>(hs + (w * T + r) * 64 + 2 * lane);
+        if (early_ptr != nullptr) {
+            er0 = ld_record(early_ptr + 2 * lane);
+            er1 = ld_record(early_ptr + 2 * lane + 1);
+        }
+        const int Kc = prm.conv_k;
+        float wA[4], wB[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int kk = j - (4 - Kc);
+            wA[j] = (kk >= 0 && vA) ? prm.conv_w[(long long)c0 * Kc + kk] : 0.f;
+            wB[j] = (kk >= 0 && vB) ? prm.conv_w[(long long)(c0 + 1) * Kc + kk] : 0.f;
+        }
+        const float bA = (prm.conv_bias != nullptr && vA) ? prm.conv_bias[c0] : 0.f;
+        const float bB = (prm.conv_bias != nullptr && vB) ? prm.conv_bias[c0 + 1] : 0.f;
+        __syncthreads();                 // every thread holds its hidden rows: the staging area may go
+        const bool act = prm.clamp_silu != 0;
+        const float tau = prm.gate_tau;
+        const bool want_mask = prm.mask != nullptr;
+        uint32_t *mrow = prm.mask + ((long long)b * L + s0) * prm.MW + g * 2;
+        const bool second_word = g * 2 + 1 < prm.MW;
+        auto phasor = [&](float u, bool valid, float &zr, float &zi) -> bool {
+            float x = u;
+            if (act) {
+                x = fminf(fmaxf(x, -50.f), 50.f);
+                x = __fdividef(x, 1.f + __expf(-x));
+            }
+            // one exponential serves both maps: with q = e^-x, sigmoid = 1/(1+q) and
+            // tanh = (1-q^2)/(1+q^2); |x| is capped where both have long saturated in fp32
+            const float xc = fminf(fmaxf(x, -25.f), 25.f);
+            const float q = __expf(-xc), q2 = q * q;
+            const float rcp = __fdividef(1.f, (1.f + q) * (1.f + q2));
+            const float m = (1.f + q2) * rcp;
+            const float th = (1.f - q2) * (1.f + q) * rcp;
+            float sn, cs;
+            __sincosf(3.14159265358979f * th, &sn, &cs);
+            // with clamp + SiLU the magnitude never falls below 0.43, and the host only admits
+            // thresholds under that: every gate is open
+            const bool open = valid && (act || u >= tau);
+            zr = open ? m * cs : 0.f;
+            zi = open ? m * sn : 0.f;
+            return open;
+        };
+#pragma unroll
+        for (int i = 0; i < T; ++i) {
+            float uA = bA, uB = bB;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                if (j >= 4 - Kc) {
+                    uA = fmaf(wA[j], hv[i + j].x, uA);
+                    uB = fmaf(wB[j], hv[i + j].y, uB);
+                }
+            }
+            float4 v;
+            const bool oA = phasor(uA, vA, v.x, v.y);
+            const bool oB = phasor(uB, vB, v.z, v.w);
+            xs[i * 32] = v;
+            if (want_mask) {
+                const unsigned bits = ((oA ? 1u : 0u) | (oB ? 2u : 0u)) << (2 * (lane & 15));
+                const unsigned w0 = __reduce_or_sync(0xffffffffu, lane < 16 ? bits : 0u);
+                const unsigned w1 = __reduce_or_sync(0xffffffffu, lane < 16 ? 0u : bits);
+                if (FULL || i < nvalid) {
+                    if (lane == 0) mrow[0] = w0;
+                    if (lane == 16 && second_word) mrow[1] = w1;
+                }
+                mrow += prm.MW;
+            }
+            if (FULL || i < nvalid) e = cfma2(a, e, v);
+        }
+    } else if constexpr (KIND == KIND_FWD) {
         // |p| >= eps decided as re^2 + im^2 >= eps^2 in double: both squares are exact there
         // and the sum rounds once, so the decision is reproducible bit for bit.  The fp32 sum
         // of squares s is within 2^-22 (relative) of the exact one, so d = s - mid, mid =
@@ -353,10 +493,8 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
             if (cpt > 0) {
                 ok = poll_pair(prm.pre + (chain * prm.KP + cpt / M) * 64, lane, epoch, prm.poll_limit,
                                mine ? er0 : none, mine ? er1 : none, r);
-            } else if (!REV && prm.state_in != nullptr) {
-                const float2 *s = prm.state_in + (long long)b * C + c0;
-                if (vA) { const float2 v = s[0]; r.x = v.x; r.y = v.y; }
-                if (vB) { const float2 v = s[1]; r.z = v.x; r.w = v.y; }
+            } else {
+                r = sinit;
             }
         }
         sm.sR[slot][lane] = r;
@@ -425,6 +563,30 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
         }
     } else if (checkpoint && w == 0) {
         publish_pair(prm.pre + (chain * prm.KP + k / M) * 64, lane, zero4(), epoch, REC_POISON);
+    }
+    if constexpr (KIND == KIND_FUSED) {
+        // the call's last conv_k-1 hidden rows (reaching back into the carried tail when the
+        // call is shorter than that) become the next call's history
+        const int Kh = prm.conv_k - 1;
+        if (prm.tail_out != nullptr && k == K - 1 && w == 0 && !failed) {
+            const float *hin = reinterpret_cast<const float *>(prm.in);
+            for (int r = 0; r < Kh; ++r) {
+                const long long t = L - Kh + r;
+                float vA_ = 0.f, vB_ = 0.f;
+                if (t >= 0) {
+                    const float *src = hin + ((long long)b * L + t) * C + c0;
+                    if (vA) vA_ = src[0];
+                    if (vB) vB_ = src[1];
+                } else if (prm.tail_in != nullptr) {
+                    const float *src = prm.tail_in + ((long long)b * Kh + (Kh + t)) * C + c0;
+                    if (vA) vA_ = src[0];
+                    if (vB) vB_ = src[1];
+                }
+                float *dst = prm.tail_out + ((long long)b * Kh + r) * C + c0;
+                if (vA) dst[0] = vA_;
+                if (vB) dst[1] = vB_;
+            }
+        }
     }
     if constexpr (KIND == KIND_BWD) {
         if (prm.qpart != nullptr) {
