@@ -154,7 +154,7 @@ CAWN_API int cawn_phase_accumulate_fwd(const cawn_params *params,
  * grad_state_out, state_in: [B,C] complex64 (device) or NULL (= 0).
  * grad_gamma, grad_theta: [C] float (device) or NULL.  grad_state_in: [B,C] complex64 or NULL.
  * Deterministic: partial sums are combined in a fixed order in double.
- * Static retention only.
+ * Static retention only (see cawn_phase_accumulate_bwd_dynamic for the other form).
  */
 CAWN_API int cawn_phase_accumulate_bwd(const cawn_params *params,
                                        const void *saved, int saved_kind,
@@ -165,6 +165,31 @@ CAWN_API int cawn_phase_accumulate_bwd(const cawn_params *params,
                                        void *grad_state_in,
                                        void *workspace, size_t workspace_bytes,
                                        void *cuda_stream);
+
+/*
+ * Backward with the paper's time-varying retention (Section "Multi-Head Dynamic Parameter
+ * Projection", item 4: gamma_{t,h,k} = sigmoid(W_gamma x_t + b_k), the projection per head and a
+ * static per-harmonic bias).  params->flags must carry CAWN_FLAG_RETENTION_DYNAMIC.
+ *   a_t = gamma_t e^{i theta},  lam_t = grad_y_t + conj(a_{t+1}) lam_{t+1}
+ *   d gamma_t(b,t,j) = Re(conj(lam_t) e^{i theta_j} P_{t-1}),  s = gamma_t (1 - gamma_t) d gamma_t
+ *   grad_gamma_logit[b,t,h] = sum_k s      grad_freq_bias[k] = sum_{b,t,h} s
+ *   grad_theta_j = sum_{b,t} Re(conj(lam_t) i a_t P_{t-1})      grad_state_in = conj(a_0) lam_0
+ * gamma_logit [B,L,H], freq_bias [F] (device).  grad_gamma_logit [B,L,H] float, grad_freq_bias [F]
+ * float, grad_theta [C] float: device or NULL.  Other arguments as cawn_phase_accumulate_bwd.
+ * grad_gamma_logit is accumulated with atomic adds (zeroed by the call first): when a head spans
+ * three or more 64-channel groups (F > 128) its last bits may differ from run to run; everything
+ * else is bitwise repeatable.
+ */
+CAWN_API int cawn_phase_accumulate_bwd_dynamic(const cawn_params *params,
+                                               const void *saved, int saved_kind,
+                                               const float *gamma_logit, const float *freq_bias,
+                                               const float *theta, const void *state_in,
+                                               const void *grad_y, const void *grad_state_out,
+                                               void *grad_p, float *grad_gamma_logit,
+                                               float *grad_freq_bias, float *grad_theta,
+                                               void *grad_state_in,
+                                               void *workspace, size_t workspace_bytes,
+                                               void *cuda_stream);
 
 /*
  * Associative combine of two segment summaries (static retention):

@@ -34,6 +34,7 @@ EXPORTS = (
     "cawn_status_string", "cawn_workspace_bytes", "cawn_workspace_init",
     "cawn_phase_accumulate_fwd", "cawn_phase_accumulate_bwd", "cawn_state_carry",
     "cawn_poll_status", "cawn_phase_accumulate_fwd_host", "cawn_phase_accumulate_fwd_static",
+    "cawn_phase_accumulate_bwd_dynamic",
 )
 
 
@@ -79,6 +80,7 @@ def lib():
         L.cawn_workspace_init.argtypes = [vp, sz, vp]
         L.cawn_phase_accumulate_fwd.argtypes = [pp, vp, fp, fp, fp, fp, fp, fp, vp, vp, vp, vp, vp, sz, vp]
         L.cawn_phase_accumulate_bwd.argtypes = [pp, vp, ctypes.c_int, fp, fp, vp, vp, vp, vp, fp, fp, vp, vp, sz, vp]
+        L.cawn_phase_accumulate_bwd_dynamic.argtypes = [pp, vp, ctypes.c_int, fp, fp, fp, vp, vp, vp, vp, fp, fp, fp, vp, vp, sz, vp]
         L.cawn_state_carry.argtypes = [pp, vp, vp, ctypes.c_int64, fp, fp, vp, vp]
         L.cawn_poll_status.argtypes = [vp, vp]
         L.cawn_phase_accumulate_fwd_host.argtypes = [pp, vp, fp, fp, vp, vp, vp, vp, vp, sz, vp]
@@ -189,3 +191,13 @@ def cawn_phase_accumulate_fwd_static(params, input, gamma, theta, y, state_in=No
         ctypes.byref(params), _dp(input), _dp(gamma), _dp(theta), _dp(state_in), _dp(y),
         _dp(state_out), _dp(gate_mask), _dp(device_status), _stream(stream)),
         "cawn_phase_accumulate_fwd_static")
+
+
+def cawn_phase_accumulate_bwd_dynamic(params, saved, saved_kind, gamma_logit, freq_bias, theta, grad_y, grad_p,
+                                      workspace, state_in=None, grad_state_out=None, grad_gamma_logit=None,
+                                      grad_freq_bias=None, grad_theta=None, grad_state_in=None, stream=None):
+    _check(lib().cawn_phase_accumulate_bwd_dynamic(
+        ctypes.byref(params), _dp(saved), saved_kind, _dp(gamma_logit), _dp(freq_bias), _dp(theta),
+        _dp(state_in), _dp(grad_y), _dp(grad_state_out), _dp(grad_p), _dp(grad_gamma_logit),
+        _dp(grad_freq_bias), _dp(grad_theta), _dp(grad_state_in), _dp(workspace),
+        workspace.numel() * workspace.element_size(), _stream(stream)), "cawn_phase_accumulate_bwd_dynamic")

@@ -99,33 +99,37 @@ inline bool grid_ok(const cawn_params *p, const Geometry &g)
 // The float4 path needs every row segment on a 16-byte boundary: C even (the arrays
 // themselves are checked to be 16-byte aligned).  The tile is staged in dynamic shared memory;
 // MINB is the number of CTAs per SM the register allocation leaves room for.
-template <int T, int W, int KIND, bool VEC, int MINB>
+template <int T, int W, int KIND, bool VEC, int MINB, bool DYN>
 cudaError_t launch_scan_inst(const ScanParams &sp, cudaStream_t st)
 {
-    constexpr size_t smem = sizeof(ScanSmem<T, W, KIND>);
+    constexpr size_t smem = sizeof(ScanSmem<T, W, KIND, DYN>);
     static bool configured[64] = {};
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= 64 || !configured[dev]) {
-        e = cudaFuncSetAttribute(cawn_scan_kernel<T, W, KIND, VEC, MINB>,
+        e = cudaFuncSetAttribute(cawn_scan_kernel<T, W, KIND, VEC, MINB, DYN>,
                                  cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) configured[dev] = true;
     }
     const dim3 grid((unsigned)sp.G, (unsigned)sp.B, (unsigned)sp.K);
-    cawn_scan_kernel<T, W, KIND, VEC, MINB><<<grid, W * 32, smem, st>>>(sp);
+    cawn_scan_kernel<T, W, KIND, VEC, MINB, DYN><<<grid, W * 32, smem, st>>>(sp);
     return cudaGetLastError();
 }
-template <int T, int W, int KIND, int MINB>
+template <int T, int W, int KIND, int MINB, bool DYN = false>
 cudaError_t launch_scan(const ScanParams &sp, cudaStream_t st)
 {
-    return sp.C % 2 == 0 ? launch_scan_inst<T, W, KIND, true, MINB>(sp, st)
-                         : launch_scan_inst<T, W, KIND, false, MINB>(sp, st);
+    return sp.C % 2 == 0 ? launch_scan_inst<T, W, KIND, true, MINB, DYN>(sp, st)
+                         : launch_scan_inst<T, W, KIND, false, MINB, DYN>(sp, st);
 }
 
-inline cudaError_t launch_fwd(TileShape ts, const ScanParams &sp, cudaStream_t st)
+inline cudaError_t launch_fwd(TileShape ts, const ScanParams &sp, cudaStream_t st, bool dyn = false)
 {
+    if (dyn) {
+        if (ts.T == 16) return launch_scan<16, 8, KIND_FWD, 2, true>(sp, st);
+        return launch_scan<4, 4, KIND_FWD, 8, true>(sp, st);
+    }
     if (ts.T == 16) return launch_scan<16, 8, KIND_FWD, 3>(sp, st);
     return launch_scan<4, 4, KIND_FWD, 8>(sp, st);
 }
@@ -134,8 +138,12 @@ inline cudaError_t launch_fused(TileShape ts, const ScanParams &sp, cudaStream_t
     if (ts.T == 16) return launch_scan<16, 8, KIND_FUSED, 3>(sp, st);
     return launch_scan<4, 4, KIND_FUSED, 8>(sp, st);
 }
-inline cudaError_t launch_bwd(TileShape ts, const ScanParams &sp, cudaStream_t st)
+inline cudaError_t launch_bwd(TileShape ts, const ScanParams &sp, cudaStream_t st, bool dyn = false)
 {
+    if (dyn) {
+        if (ts.T == 8) return launch_scan<8, 8, KIND_BWD, 2, true>(sp, st);
+        return launch_scan<4, 4, KIND_BWD, 8, true>(sp, st);
+    }
     if (ts.T == 8) return launch_scan<8, 8, KIND_BWD, 3>(sp, st);
     return launch_scan<4, 4, KIND_BWD, 8>(sp, st);
 }
@@ -220,6 +228,7 @@ int cawn_workspace_bytes(const cawn_params *params, int op, size_t *bytes)
         size_t rec = gb.rec_bytes > gf.rec_bytes ? gb.rec_bytes : gf.rec_bytes;
         size_t total = sizeof(WsHeader) + round_up(rec, 256);
         total += round_up((size_t)params->B * gb.K * gb.C * sizeof(float2), 256);
+        total += round_up((size_t)params->B * gb.K * gb.C * sizeof(float), 256);
         if (op == CAWN_OP_BWD_PUSHES) total += round_up(n * sizeof(float2), 256);
         *bytes = total;
         return CAWN_OK;
@@ -255,9 +264,13 @@ int cawn_phase_accumulate_fwd(const cawn_params *params, const void *input,
 {
     int rc = check_params(params);
     if (rc != CAWN_OK) return rc;
-    (void)gamma_logit; (void)freq_bias;
-    if (params->flags & CAWN_FLAG_RETENTION_DYNAMIC) return CAWN_ERR_UNSUPPORTED;
+    const bool dyn = (params->flags & CAWN_FLAG_RETENTION_DYNAMIC) != 0;
     const bool fused = params->conv_k != 0;
+    if (dyn) {
+        if (fused) return CAWN_ERR_UNSUPPORTED;
+        if (gamma_logit == nullptr || freq_bias == nullptr) return CAWN_ERR_NULL_POINTER;
+        if (!aligned(gamma_logit, 4) || !aligned(freq_bias, 4)) return CAWN_ERR_MISALIGNED;
+    }
     if (fused) {
         if (params->conv_k > 4) return CAWN_ERR_UNSUPPORTED;
         if (conv_w == nullptr) return CAWN_ERR_NULL_POINTER;
@@ -266,7 +279,7 @@ int cawn_phase_accumulate_fwd(const cawn_params *params, const void *input,
         if ((params->flags & CAWN_FLAG_PRELUDE_CLAMP_SILU) && params->gate_eps > 0.4f) return CAWN_ERR_UNSUPPORTED;
         if (!aligned(conv_w, 4) || !aligned(conv_bias, 4)) return CAWN_ERR_MISALIGNED;
     }
-    if (gamma == nullptr || theta == nullptr || workspace == nullptr) return CAWN_ERR_NULL_POINTER;
+    if ((gamma == nullptr && !dyn) || theta == nullptr || workspace == nullptr) return CAWN_ERR_NULL_POINTER;
     if (params->L > 0 && (input == nullptr || y == nullptr)) return CAWN_ERR_NULL_POINTER;
     if (!aligned(input, 16) || !aligned(y, 16) || !aligned(workspace, 16) ||
         !aligned(gate_mask, 4) || !aligned(state_in, 8) || !aligned(state_out, 8) ||
@@ -315,24 +328,29 @@ int cawn_phase_accumulate_fwd(const cawn_params *params, const void *input,
         if (launch_fused(ts, sp, st) != cudaSuccess) return CAWN_ERR_CUDA;
         return CAWN_OK;
     }
-    if (launch_fwd(ts, sp, st) != cudaSuccess) return CAWN_ERR_CUDA;
+    sp.gamma_logit = gamma_logit; sp.freq_bias = freq_bias; sp.H = params->H; sp.F = params->F;
+    if (launch_fwd(ts, sp, st, dyn) != cudaSuccess) return CAWN_ERR_CUDA;
     return CAWN_OK;
 }
 
-int cawn_phase_accumulate_bwd(const cawn_params *params, const void *saved, int saved_kind,
-                              const float *gamma, const float *theta, const void *state_in,
-                              const void *grad_y, const void *grad_state_out,
-                              void *grad_p, float *grad_gamma, float *grad_theta,
-                              void *grad_state_in, void *workspace, size_t workspace_bytes,
-                              void *cuda_stream)
+// Backward of the Cartesian forward, static (gamma) or time-varying (gamma_logit, freq_bias)
+// retention.  Static: grad_gamma; time-varying: grad_logit [B,L,H], grad_fbias [F].
+static int bwd_common(const cawn_params *params, bool dyn, const void *saved, int saved_kind,
+                      const float *gamma, const float *gamma_logit, const float *freq_bias,
+                      const float *theta, const void *state_in,
+                      const void *grad_y, const void *grad_state_out,
+                      void *grad_p, float *grad_gamma, float *grad_logit, float *grad_fbias,
+                      float *grad_theta, void *grad_state_in, void *workspace, size_t workspace_bytes,
+                      void *cuda_stream)
 {
     int rc = check_params(params);
     if (rc != CAWN_OK) return rc;
-    if (params->conv_k != 0 || (params->flags & CAWN_FLAG_RETENTION_DYNAMIC))
-        return CAWN_ERR_UNSUPPORTED;
+    if (params->conv_k != 0) return CAWN_ERR_UNSUPPORTED;
     if (saved_kind != CAWN_SAVED_STATES && saved_kind != CAWN_SAVED_PUSHES) return CAWN_ERR_INVALID_ARG;
-    if (gamma == nullptr || theta == nullptr || workspace == nullptr) return CAWN_ERR_NULL_POINTER;
-    const bool want_param = (grad_gamma != nullptr || grad_theta != nullptr);
+    if (theta == nullptr || workspace == nullptr) return CAWN_ERR_NULL_POINTER;
+    if (dyn ? (gamma_logit == nullptr || freq_bias == nullptr) : gamma == nullptr) return CAWN_ERR_NULL_POINTER;
+    const bool want_param = (grad_gamma != nullptr || grad_theta != nullptr || grad_logit != nullptr ||
+                             grad_fbias != nullptr);
     if (params->L > 0 && (grad_y == nullptr || grad_p == nullptr)) return CAWN_ERR_NULL_POINTER;
     if (params->L > 0 && want_param && saved == nullptr) return CAWN_ERR_NULL_POINTER;
     if (!aligned(saved, 16) || !aligned(grad_y, 16) || !aligned(grad_p, 16) || !aligned(workspace, 16) ||
@@ -357,14 +375,20 @@ int cawn_phase_accumulate_bwd(const cawn_params *params, const void *saved, int 
         }
         if (grad_gamma && cudaMemsetAsync(grad_gamma, 0, C * sizeof(float), st) != cudaSuccess) return CAWN_ERR_CUDA;
         if (grad_theta && cudaMemsetAsync(grad_theta, 0, C * sizeof(float), st) != cudaSuccess) return CAWN_ERR_CUDA;
+        if (grad_fbias && cudaMemsetAsync(grad_fbias, 0, params->F * sizeof(float), st) != cudaSuccess) return CAWN_ERR_CUDA;
         return CAWN_OK;
     }
+    // the logit gradient is accumulated with atomic adds: it starts from zero
+    if (grad_logit != nullptr &&
+        cudaMemsetAsync(grad_logit, 0, (size_t)params->B * (size_t)params->L * params->H * sizeof(float), st) != cudaSuccess)
+        return CAWN_ERR_CUDA;
 
     char *base = reinterpret_cast<char *>(workspace);
     const size_t rec = gb.rec_bytes > gf.rec_bytes ? gb.rec_bytes : gf.rec_bytes;
     size_t off = sizeof(WsHeader);
     char *recs = base + off;                                        off += round_up(rec, 256);
     float2 *qpart = reinterpret_cast<float2 *>(base + off);         off += round_up((size_t)params->B * gb.K * C * sizeof(float2), 256);
+    float *spart = reinterpret_cast<float *>(base + off);           off += round_up((size_t)params->B * gb.K * C * sizeof(float), 256);
     float2 *Pbuf = reinterpret_cast<float2 *>(base + off);
 
     const void *states = saved;
@@ -381,7 +405,8 @@ int cawn_phase_accumulate_bwd(const cawn_params *params, const void *saved, int 
         set_gate(fp, params->gate_eps);
         fp.clampv = 0.f;
         fp.poll_limit = kPollLimit;
-        if (launch_fwd(tf, fp, st) != cudaSuccess) return CAWN_ERR_CUDA;
+        fp.gamma_logit = gamma_logit; fp.freq_bias = freq_bias; fp.H = params->H; fp.F = params->F;
+        if (launch_fwd(tf, fp, st, dyn) != cudaSuccess) return CAWN_ERR_CUDA;
         states = Pbuf;
     }
 
@@ -399,15 +424,50 @@ int cawn_phase_accumulate_bwd(const cawn_params *params, const void *saved, int 
     sp.L = params->L; sp.B = params->B;
     sp.clampv = params->grad_clamp_abs > 0.f ? params->grad_clamp_abs : 0.f;
     sp.poll_limit = kPollLimit;
-    if (launch_bwd(tb, sp, st) != cudaSuccess) return CAWN_ERR_CUDA;
+    sp.gamma_logit = gamma_logit; sp.freq_bias = freq_bias; sp.H = params->H; sp.F = params->F;
+    sp.grad_logit = (dyn && want_param) ? grad_logit : nullptr;
+    sp.spart = (dyn && want_param && grad_fbias != nullptr) ? spart : nullptr;
+    if (launch_bwd(tb, sp, st, dyn) != cudaSuccess) return CAWN_ERR_CUDA;
 
     if (want_param) {
         const int warps = 8;
         cawn_bwd_finalize_kernel<<<(C + warps - 1) / warps, warps * 32, 0, st>>>(
-            qpart, params->B * gb.K, C, gamma, theta, grad_gamma, grad_theta, sp.clampv);
+            qpart, params->B * gb.K, C, dyn ? nullptr : gamma, theta, dyn ? nullptr : grad_gamma, grad_theta, sp.clampv);
         if (cudaGetLastError() != cudaSuccess) return CAWN_ERR_CUDA;
+        if (dyn && grad_fbias != nullptr) {
+            cawn_bwd_freq_bias_kernel<<<(params->F + warps - 1) / warps, warps * 32, 0, st>>>(
+                spart, params->B * gb.K, params->H, params->F, grad_fbias);
+            if (cudaGetLastError() != cudaSuccess) return CAWN_ERR_CUDA;
+        }
     }
     return CAWN_OK;
+}
+
+int cawn_phase_accumulate_bwd(const cawn_params *params, const void *saved, int saved_kind,
+                              const float *gamma, const float *theta, const void *state_in,
+                              const void *grad_y, const void *grad_state_out,
+                              void *grad_p, float *grad_gamma, float *grad_theta,
+                              void *grad_state_in, void *workspace, size_t workspace_bytes,
+                              void *cuda_stream)
+{
+    if (params != nullptr && (params->flags & CAWN_FLAG_RETENTION_DYNAMIC)) return CAWN_ERR_UNSUPPORTED;
+    return bwd_common(params, false, saved, saved_kind, gamma, nullptr, nullptr, theta, state_in, grad_y,
+                      grad_state_out, grad_p, grad_gamma, nullptr, nullptr, grad_theta, grad_state_in,
+                      workspace, workspace_bytes, cuda_stream);
+}
+
+int cawn_phase_accumulate_bwd_dynamic(const cawn_params *params, const void *saved, int saved_kind,
+                                      const float *gamma_logit, const float *freq_bias,
+                                      const float *theta, const void *state_in,
+                                      const void *grad_y, const void *grad_state_out,
+                                      void *grad_p, float *grad_gamma_logit, float *grad_freq_bias,
+                                      float *grad_theta, void *grad_state_in,
+                                      void *workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    if (params != nullptr && !(params->flags & CAWN_FLAG_RETENTION_DYNAMIC)) return CAWN_ERR_INVALID_ARG;
+    return bwd_common(params, true, saved, saved_kind, nullptr, gamma_logit, freq_bias, theta, state_in, grad_y,
+                      grad_state_out, grad_p, nullptr, grad_gamma_logit, grad_freq_bias, grad_theta,
+                      grad_state_in, workspace, workspace_bytes, cuda_stream);
 }
 
 int cawn_state_carry(const cawn_params *params, const void *state_prev, const void *state_local,

@@ -141,4 +141,51 @@ __device__ __forceinline__ bool poll_pair(const uint4 *tile_recs, int lane, unsi
     }
 }
 
+// ---------------------------------------------------------------------------------------
+// Time-varying retention: one step is  P <- g (a P) + x  with a real per-step factor g per
+// channel on top of the fixed rotation a; a segment is summarised by its end state and the
+// product of its factors.
+__device__ __forceinline__ float4 scale_step2(float4 a, float4 P, float2 g, float4 x)
+{
+    const float4 t = cmul2(a, P);
+    return make_float4(fmaf(g.x, t.x, x.x), fmaf(g.x, t.y, x.y), fmaf(g.y, t.z, x.z), fmaf(g.y, t.w, x.w));
+}
+__device__ __forceinline__ float sigmoidf_fast(float s) { return __fdividef(1.f, 1.f + __expf(-s)); }
+
+// Records of the time-varying form: {re, im, factor product, tag} with a 32-bit tag
+// (epoch mod 2^30) * 4 + kind.
+__device__ __forceinline__ unsigned record_kind32(uint4 r, unsigned long long epoch)
+{
+    return (r.w >> 2) == (unsigned)(epoch & 0x3fffffffull) ? (r.w & 3u) : 0u;
+}
+__device__ __forceinline__ void publish_pair_d(uint4 *tile_recs, int lane, float4 v, float2 d,
+                                               unsigned long long epoch, unsigned kind)
+{
+    const unsigned tag = (unsigned)(epoch & 0x3fffffffull) * 4u + kind;
+    uint4 *p = tile_recs + 2 * lane;
+    asm volatile("st.relaxed.gpu.global.v4.u32 [%0], {%1, %2, %3, %4};"
+                 :: "l"(p), "r"(__float_as_uint(v.x)), "r"(__float_as_uint(v.y)), "r"(__float_as_uint(d.x)), "r"(tag) : "memory");
+    asm volatile("st.relaxed.gpu.global.v4.u32 [%0], {%1, %2, %3, %4};"
+                 :: "l"(p + 1), "r"(__float_as_uint(v.z)), "r"(__float_as_uint(v.w)), "r"(__float_as_uint(d.y)), "r"(tag) : "memory");
+}
+__device__ __forceinline__ bool poll_pair_d(const uint4 *tile_recs, int lane, unsigned long long epoch,
+                                            unsigned poll_limit, uint4 r0, uint4 r1, float4 &v, float2 &d)
+{
+    const uint4 *p = tile_recs + 2 * lane;
+    unsigned polls = 0;
+    for (;;) {
+        const unsigned k0 = record_kind32(r0, epoch), k1 = record_kind32(r1, epoch);
+        if (k0 != 0u && k1 != 0u) {
+            v = make_float4(__uint_as_float(r0.x), __uint_as_float(r0.y),
+                            __uint_as_float(r1.x), __uint_as_float(r1.y));
+            d = make_float2(__uint_as_float(r0.z), __uint_as_float(r1.z));
+            return k0 != REC_POISON && k1 != REC_POISON;
+        }
+        if (++polls > poll_limit) { v = zero4(); d = make_float2(0.f, 0.f); return false; }
+        if (polls > 4) __nanosleep(polls > 64 ? 256 : 32);
+        r0 = ld_record(p);
+        r1 = ld_record(p + 1);
+    }
+}
+
 }  // namespace cawn

@@ -79,11 +79,17 @@ struct ScanParams {
     int conv_k;                  // 1..4
     int clamp_silu;              // clamp the conv output to +-50, then SiLU
     float gate_tau;              // gate: conv output >= gate_tau (fp32 fmaf chain, tap order)
+    // time-varying retention (DYN): gamma_t = sigmoid(gamma_logit[b,t,h] + freq_bias[k])
+    const float *gamma_logit;    // [B][L][H]
+    const float *freq_bias;      // [F]
+    int H, F;
+    float *grad_logit;           // BWD: [B][L][H], zeroed before the launch (atomic adds)
+    float *spart;                // BWD: per-tile partial sums of the logit gradient [B*K][C]
 };
 
 // Shared memory of one CTA: the tile (two tiles in the backward: grad_y and P_{t-1}), then the
 // small exchange areas.
-template <int T, int W, int KIND>
+template <int T, int W, int KIND, bool DYN = false>
 struct ScanSmem {
     static constexpr int TILE = T * W;
     static constexpr int NT = (KIND == KIND_BWD) ? 2 : 1;
@@ -91,6 +97,8 @@ struct ScanSmem {
     float4 sE[W][32];
     float4 sR[kWindow + 1][32];
     float sCoef[64][6];
+    float2 sD[DYN ? W : 1][DYN ? 32 : 1];             // DYN: factor products of the warps' steps
+    float2 sRD[DYN ? kWindow + 1 : 1][DYN ? 32 : 1];  // DYN: factor products of the window's tiles
     unsigned long long epoch;
     int err;
     int pad;
@@ -157,10 +165,11 @@ __device__ __forceinline__ void fetch_rows(float4 *dst, uint32_t dst_s, const ch
     }
 }
 
-template <int T, int W, int KIND, bool VEC, bool FULL>
-__device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, KIND> &sm,
+template <int T, int W, int KIND, bool VEC, bool DYN, bool FULL>
+__device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, KIND, DYN> &sm,
                                           const int g, const int b, const int k)
 {
+    static_assert(!(DYN && KIND == KIND_FUSED), "time-varying retention is not built for the fused path");
     constexpr bool REV = (KIND == KIND_BWD);
     constexpr int TILE = T * W;
     constexpr int M = kWindow;
@@ -244,7 +253,7 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
         float re = 0.f, im = 0.f;
         if (ch < C) {
             const int n = task == 0 ? 1 : (task == 1 ? T : TILE);
-            const double gm = (double)prm.gamma[ch], th = (double)prm.theta[ch];
+            const double gm = DYN ? 1.0 : (double)prm.gamma[ch], th = (double)prm.theta[ch];
             double mag = 1.0, base = gm;
             for (int m = n; m > 0; m >>= 1) {            // gamma^n by square-and-multiply
                 if (m & 1) mag *= base;
@@ -278,6 +287,26 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
         aT = make_float4(u0.z, u0.w, u2.x, u2.y);
     }
     const unsigned long long epoch = sm.epoch;
+
+    // Time-varying retention: this lane's heads and per-harmonic biases, and the factor pair of
+    // one physical row t (0 outside the call, which only ever multiplies a zero carry).
+    int hA = 0, hB = 0;
+    float fbA = 0.f, fbB = 0.f;
+    if constexpr (DYN) {
+        hA = c0 / prm.F; hB = (c0 + 1) / prm.F;
+        if (vA) fbA = prm.freq_bias[c0 % prm.F];
+        if (vB) fbB = prm.freq_bias[(c0 + 1) % prm.F];
+    }
+    auto row_gamma = [&](long long t) -> float2 {
+        float2 gm = make_float2(0.f, 0.f);
+        if (t >= 0 && t < L) {
+            const float *gl = prm.gamma_logit + ((long long)b * L + t) * prm.H;
+            if (vA) gm.x = sigmoidf_fast(gl[hA] + fbA);
+            if (vB) gm.y = sigmoidf_fast(gl[hB] + fbB);
+        }
+        return gm;
+    };
+    float2 dprod = make_float2(1.f, 1.f);                // product of this thread's step factors
 
     // Window of carry records this tile needs (see the header comment), and a first,
     // non-blocking reading of the record this warp is responsible for: it is usually there
@@ -412,6 +441,7 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
             float nearest = INFINITY;
             uint32_t *mrow = mrow0;
             e = zero4();
+            dprod = make_float2(1.f, 1.f);
 #pragma unroll
             for (int i = 0; i < T; ++i) {
                 if (!EXACT && i % GR == 0) {
@@ -446,7 +476,15 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
                     }
                     mrow += prm.MW;
                 }
-                if (FULL || i < nvalid) e = cfma2(a, e, v);
+                if (FULL || i < nvalid) {
+                    if constexpr (DYN) {
+                        const float2 gm = row_gamma(s0 + i);
+                        e = scale_step2(a, e, gm, v);
+                        dprod.x *= gm.x; dprod.y *= gm.y;
+                    } else {
+                        e = cfma2(a, e, v);
+                    }
+                }
             }
             return nearest;
         };
@@ -461,11 +499,26 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
             er0 = ld_record(early_ptr + 2 * lane);
             er1 = ld_record(early_ptr + 2 * lane + 1);
         }
+        if constexpr (DYN) {
+            // moving from row t+1 to row t multiplies by gamma_{t+1} conj(R): the factor of the
+            // row processed just before (row L does not exist: factor 0 on a zero carry)
+            float2 gm = row_gamma(t_first + 1);
 #pragma unroll
-        for (int i = 0; i < T; ++i)
-            if (FULL || i < nvalid) e = cfma2(a, e, xs[i * 32]);
+            for (int i = 0; i < T; ++i) {
+                if (FULL || i < nvalid) {
+                    e = scale_step2(a, e, gm, xs[i * 32]);
+                    dprod.x *= gm.x; dprod.y *= gm.y;
+                    gm = row_gamma(t_first - i);
+                }
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < T; ++i)
+                if (FULL || i < nvalid) e = cfma2(a, e, xs[i * 32]);
+        }
     }
     sm.sE[w][lane] = e;
+    if constexpr (DYN) sm.sD[w][lane] = dprod;
     if (tid == 0 && arrived == gridDim.x * gridDim.y * gridDim.z - 1) {
         // every CTA of this launch has read the epoch: open the next one
         st_volatile_u32(&prm.ws->done, 0u);
@@ -476,9 +529,20 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
     // ---- 2. publish the aggregate, fetch the carry window ----------------------------------
     if (w == 0 && k + 1 < K) {
         float4 E = sm.sE[0][lane];
+        if constexpr (DYN) {
+            float2 D = sm.sD[0][lane];
 #pragma unroll
-        for (int i = 1; i < W; ++i) E = cfma2(aT, E, sm.sE[i][lane]);
-        publish_pair(prm.agg + (chain * K + k) * 64, lane, E, epoch, REC_AGGREGATE);
+            for (int i = 1; i < W; ++i) {
+                const float2 di = sm.sD[i][lane];
+                E = scale_step2(aT, E, di, sm.sE[i][lane]);
+                D.x *= di.x; D.y *= di.y;
+            }
+            publish_pair_d(prm.agg + (chain * K + k) * 64, lane, E, D, epoch, REC_AGGREGATE);
+        } else {
+#pragma unroll
+            for (int i = 1; i < W; ++i) E = cfma2(aT, E, sm.sE[i][lane]);
+            publish_pair(prm.agg + (chain * K + k) * 64, lane, E, epoch, REC_AGGREGATE);
+        }
     }
     // slot r < nrec of the window: aggregate of tile k-1-r; slot M: the carry-in the window starts from
     for (int slot = w; slot <= M; slot += W) {
@@ -486,18 +550,22 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
         bool ok = true;
         const uint4 none = make_uint4(0u, 0u, 0u, 0u);
         const bool mine = (slot == w);                   // the slot read ahead of phase 1
+        float2 rd = make_float2(0.f, 0.f);
         if (slot < nrec) {
-            ok = poll_pair(prm.agg + (chain * K + (k - 1 - slot)) * 64, lane, epoch, prm.poll_limit,
-                           mine ? er0 : none, mine ? er1 : none, r);
+            const uint4 *rec = prm.agg + (chain * K + (k - 1 - slot)) * 64;
+            if constexpr (DYN) ok = poll_pair_d(rec, lane, epoch, prm.poll_limit, mine ? er0 : none, mine ? er1 : none, r, rd);
+            else ok = poll_pair(rec, lane, epoch, prm.poll_limit, mine ? er0 : none, mine ? er1 : none, r);
         } else if (slot == M) {
             if (cpt > 0) {
-                ok = poll_pair(prm.pre + (chain * prm.KP + cpt / M) * 64, lane, epoch, prm.poll_limit,
-                               mine ? er0 : none, mine ? er1 : none, r);
+                const uint4 *rec = prm.pre + (chain * prm.KP + cpt / M) * 64;
+                if constexpr (DYN) ok = poll_pair_d(rec, lane, epoch, prm.poll_limit, mine ? er0 : none, mine ? er1 : none, r, rd);
+                else ok = poll_pair(rec, lane, epoch, prm.poll_limit, mine ? er0 : none, mine ? er1 : none, r);
             } else {
                 r = sinit;
             }
         }
         sm.sR[slot][lane] = r;
+        if constexpr (DYN) sm.sRD[slot][lane] = rd;
         if (!ok) {
             sm.err = 1;
             atomicMax(&prm.ws->status, 1u);              // CAWN_ERR_CARRY_TIMEOUT
@@ -509,6 +577,7 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
     const bool failed = (sm.err != 0);
     const bool checkpoint = (k > 0 && k % M == 0 && k + 1 < K);
     float4 qa = zero4();
+    float2 sacc_out = make_float2(0.f, 0.f);
     if (!failed) {
         float4 P = sm.sR[M][lane];
         {
@@ -516,18 +585,37 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
             const float4 u1 = cp[1], u2 = cp[2];
             const float4 AA = make_float4(u1.x, u1.y, u2.z, u2.w);
 #pragma unroll 1
-            for (int i = nrec - 1; i >= 0; --i) P = cfma2(AA, P, sm.sR[i][lane]);
+            for (int i = nrec - 1; i >= 0; --i) {
+                if constexpr (DYN) P = scale_step2(AA, P, sm.sRD[i][lane], sm.sR[i][lane]);
+                else P = cfma2(AA, P, sm.sR[i][lane]);
+            }
         }
-        if (checkpoint && w == 0)
-            publish_pair(prm.pre + (chain * prm.KP + k / M) * 64, lane, P, epoch, REC_PREFIX);
+        if (checkpoint && w == 0) {
+            if constexpr (DYN) publish_pair_d(prm.pre + (chain * prm.KP + k / M) * 64, lane, P, make_float2(0.f, 0.f), epoch, REC_PREFIX);
+            else publish_pair(prm.pre + (chain * prm.KP + k / M) * 64, lane, P, epoch, REC_PREFIX);
+        }
 #pragma unroll 1
-        for (int i = 0; i < w; ++i) P = cfma2(aT, P, sm.sE[i][lane]);
+        for (int i = 0; i < w; ++i) {
+            if constexpr (DYN) P = scale_step2(aT, P, sm.sD[i][lane], sm.sE[i][lane]);
+            else P = cfma2(aT, P, sm.sE[i][lane]);
+        }
 
         char *r = reinterpret_cast<char *>(prm.out) + e0 * 8;
         const float cl = prm.clampv;
+        // DYN: factor of the step into row i (forward: the row's own; backward: the factor of
+        // the row processed before it), and the running sum of the logit gradient
+        float2 gstep = make_float2(0.f, 0.f), sacc = make_float2(0.f, 0.f);
+        if constexpr (DYN && REV) gstep = row_gamma(t_first + 1);
         auto step_row = [&](int i, bool clamped) {
             if (FULL || i < nvalid) {
-                P = cfma2(a, P, xs[i * 32]);
+                float2 gown = make_float2(0.f, 0.f);
+                if constexpr (DYN) {
+                    if (!REV) gstep = row_gamma(s0 + i);
+                    P = scale_step2(a, P, gstep, xs[i * 32]);
+                    if (REV) { gown = row_gamma(t_first - i); gstep = gown; }
+                } else {
+                    P = cfma2(a, P, xs[i * 32]);
+                }
                 const float4 o = clamped ? clamp4(P, cl) : P;
                 if (VEC) {
                     if (vA) __stcs(reinterpret_cast<float4 *>(r), o);
@@ -539,10 +627,38 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
                 if constexpr (KIND == KIND_BWD) {
                     // conj(lam) * P_{t-1}
                     const float4 q = sm.tile[1][w * T + i][lane];
-                    qa.x = fmaf(P.x, q.x, fmaf(P.y, q.y, qa.x));
-                    qa.y = fmaf(P.x, q.y, fmaf(-P.y, q.x, qa.y));
-                    qa.z = fmaf(P.z, q.z, fmaf(P.w, q.w, qa.z));
-                    qa.w = fmaf(P.z, q.w, fmaf(-P.w, q.z, qa.w));
+                    if constexpr (DYN) {
+                        if (prm.aux != nullptr) {
+                            // u = conj(lam_t) P_{t-1};  d gamma_t = Re(e^{i theta} u), chained through the
+                            // sigmoid; the rotation gradient sums gamma_t u
+                            const float uAx = fmaf(P.x, q.x, P.y * q.y), uAy = fmaf(P.x, q.y, -P.y * q.x);
+                            const float uBx = fmaf(P.z, q.z, P.w * q.w), uBy = fmaf(P.z, q.w, -P.w * q.z);
+                            qa.x = fmaf(gown.x, uAx, qa.x); qa.y = fmaf(gown.x, uAy, qa.y);
+                            qa.z = fmaf(gown.y, uBx, qa.z); qa.w = fmaf(gown.y, uBy, qa.w);
+                            // a holds conj(e^{i theta}) in the backward
+                            const float sA = gown.x * (1.f - gown.x) * fmaf(a.x, uAx, a.y * uAy);
+                            const float sB = gown.y * (1.f - gown.y) * fmaf(a.z, uBx, a.w * uBy);
+                            sacc.x += sA; sacc.y += sB;
+                            if (prm.grad_logit != nullptr) {
+                                // sum over the harmonics of each head present in this 64-channel group
+                                const int h_lo = (g * 64) / prm.F;
+                                const int c_hi = g * 64 + 63 < C - 1 ? g * 64 + 63 : C - 1;
+                                const int h_hi = c_hi / prm.F;
+                                for (int h = h_lo; h <= h_hi; ++h) {
+                                    float v = (vA && hA == h ? sA : 0.f) + (vB && hB == h ? sB : 0.f);
+#pragma unroll
+                                    for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+                                    if (lane == 0)
+                                        atomicAdd(prm.grad_logit + ((long long)b * L + (t_first - i)) * prm.H + h, v);
+                                }
+                            }
+                        }
+                    } else {
+                        qa.x = fmaf(P.x, q.x, fmaf(P.y, q.y, qa.x));
+                        qa.y = fmaf(P.x, q.y, fmaf(-P.y, q.x, qa.y));
+                        qa.z = fmaf(P.z, q.z, fmaf(P.w, q.w, qa.z));
+                        qa.w = fmaf(P.z, q.w, fmaf(-P.w, q.z, qa.w));
+                    }
                 }
             }
             r += rowbytes;
@@ -554,15 +670,20 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
 #pragma unroll
             for (int i = 0; i < T; ++i) step_row(i, false);
         }
+        sacc_out = sacc;
         // the thread that owns the last step writes the carried state (never clamped)
         if (prm.state_out != nullptr && nvalid > 0 && s0 + nvalid == L) {
-            if (REV) P = cmul2(a, P);                    // grad_state_in = conj(a) lam_0
+            if (REV) {                                   // grad_state_in = conj(a_0) lam_0
+                P = cmul2(a, P);
+                if constexpr (DYN) { P.x *= gstep.x; P.y *= gstep.x; P.z *= gstep.y; P.w *= gstep.y; }
+            }
             float2 *s = prm.state_out + (long long)b * C + c0;
             if (vA) s[0] = make_float2(P.x, P.y);
             if (vB) s[1] = make_float2(P.z, P.w);
         }
     } else if (checkpoint && w == 0) {
-        publish_pair(prm.pre + (chain * prm.KP + k / M) * 64, lane, zero4(), epoch, REC_POISON);
+        if constexpr (DYN) publish_pair_d(prm.pre + (chain * prm.KP + k / M) * 64, lane, zero4(), make_float2(0.f, 0.f), epoch, REC_POISON);
+        else publish_pair(prm.pre + (chain * prm.KP + k / M) * 64, lane, zero4(), epoch, REC_POISON);
     }
     if constexpr (KIND == KIND_FUSED) {
         // the call's last conv_k-1 hidden rows (reaching back into the carried tail when the
@@ -604,24 +725,38 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
                 if (vA) qp[0] = make_float2(acc.x, acc.y);
                 if (vB) qp[1] = make_float2(acc.z, acc.w);
             }
+            if constexpr (DYN) {
+                if (prm.spart != nullptr) {
+                    sm.sD[w][lane] = sacc_out;
+                    __syncthreads();
+                    if (w == 0) {
+                        float2 acc = sm.sD[0][lane];
+#pragma unroll
+                        for (int i = 1; i < W; ++i) { const float2 v = sm.sD[i][lane]; acc.x += v.x; acc.y += v.y; }
+                        float *sp = prm.spart + ((long long)b * K + k) * C + c0;
+                        if (vA) sp[0] = acc.x;
+                        if (vB) sp[1] = acc.y;
+                    }
+                }
+            }
         }
     }
 }
 
-template <int T, int W, int KIND, bool VEC, int MINB>
+template <int T, int W, int KIND, bool VEC, int MINB, bool DYN = false>
 __global__ void __launch_bounds__(W * 32, MINB) cawn_scan_kernel(const ScanParams prm)
 {
     constexpr int TILE = T * W;
     extern __shared__ __align__(128) unsigned char smem_raw[];
-    ScanSmem<T, W, KIND> &sm = *reinterpret_cast<ScanSmem<T, W, KIND> *>(smem_raw);
+    ScanSmem<T, W, KIND, DYN> &sm = *reinterpret_cast<ScanSmem<T, W, KIND, DYN> *>(smem_raw);
 
     // grid = (G, B, K): blocks are dispatched x fastest, so a tile's predecessors along time
     // (smaller k) always have smaller linear block indices
     const int g = blockIdx.x, b = blockIdx.y;
     const int k = blockIdx.z;                         // tile index along (logical) time
     const bool full = ((long long)(k + 1) * TILE <= prm.L) && (g * 64 + 64 <= prm.C);
-    if (full) scan_tile<T, W, KIND, VEC, true>(prm, sm, g, b, k);
-    else      scan_tile<T, W, KIND, VEC, false>(prm, sm, g, b, k);
+    if (full) scan_tile<T, W, KIND, VEC, DYN, true>(prm, sm, g, b, k);
+    else      scan_tile<T, W, KIND, VEC, DYN, false>(prm, sm, g, b, k);
 }
 
 // grad_gamma_j = Re(e^{i theta} Q_j), grad_theta_j = -Im(a_j Q_j), Q_j = sum of the per-tile
@@ -645,7 +780,7 @@ __global__ void cawn_bwd_finalize_kernel(const float2 *qpart, int nparts, int C,
         si += __shfl_down_sync(0xffffffffu, si, off);
     }
     if (lane == 0) {
-        const double gm = (double)gamma[ch];
+        const double gm = gamma != nullptr ? (double)gamma[ch] : 1.0;   // time-varying: already in Q
         double sn, cs;
         sincos((double)theta[ch], &sn, &cs);
         double dg = cs * sr - sn * si;
@@ -654,6 +789,24 @@ __global__ void cawn_bwd_finalize_kernel(const float2 *qpart, int nparts, int C,
         if (grad_gamma != nullptr) grad_gamma[ch] = (float)dg;
         if (grad_theta != nullptr) grad_theta[ch] = (float)dth;
     }
+}
+
+// Time-varying retention: grad_freq_bias[k] = sum over tiles and heads of the per-channel
+// partial sums of the logit gradient, in a fixed order, in double.  One warp per harmonic.
+__global__ void cawn_bwd_freq_bias_kernel(const float *spart, int nparts, int H, int F, float *grad_freq_bias)
+{
+    const int lane = threadIdx.x & 31;
+    const int kf = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (kf >= F) return;
+    const long long C = (long long)H * F;
+    double acc = 0.0;
+    for (long long i = lane; i < (long long)nparts * H; i += 32) {
+        const long long part = i / H, h = i % H;
+        acc += (double)spart[part * C + h * F + kf];
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) acc += __shfl_down_sync(0xffffffffu, acc, off);
+    if (lane == 0) grad_freq_bias[kf] = (float)acc;
 }
 
 // state_out = a^n * state_prev + state_local with a^n = gamma^n (cos n theta, sin n theta)
