@@ -161,7 +161,8 @@ def run_ours(args):
     B, L, C = cfg.B, cfg.L, cfg.C
     tokens = B * L
     nelem = tokens * C
-    prm = cb.make_params(B, L, cfg.H, cfg.F, gate_eps=cfg.gate_eps)
+    # every step reads a buffer set that no earlier step writes: the calls may overlap their tails
+    prm = cb.make_params(B, L, cfg.H, cfg.F, gate_eps=cfg.gate_eps, flags=cb.CAWN_FLAG_INPUT_INDEPENDENT)
     d = inputs.scan_inputs(B, L, C, cfg.seed + 1000 * rank, cfg.gamma_lo, cfg.gamma_hi)
     gamma = torch.from_numpy(d["gamma"]).cuda()
     theta = torch.from_numpy(d["theta"]).cuda()
@@ -188,14 +189,15 @@ def run_ours(args):
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
-    ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
-    ev[0].record(stream)
+    # two events bracket the K steps: an event between two launches would make each launch wait for
+    # the one before to drain completely, which back-to-back calls on a stream do not do
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record(stream)
     for i in range(args.steps):
         step(args.warmup + i)
-        ev[i + 1].record(stream)
+    ev1.record(stream)
     barrier()
-    total_ms = ev[0].elapsed_time(ev[-1])
-    per = sorted(ev[i].elapsed_time(ev[i + 1]) for i in range(args.steps))
+    total_ms = ev0.elapsed_time(ev1)
     status = cb.cawn_poll_status(ws)
     if status != 0:
         raise RuntimeError("device status: " + cb.status_string(status))
@@ -246,7 +248,6 @@ def run_ours(args):
                        "l2": "steps rotate over %d buffer sets (%.2f GB) > 126 MB L2"
                              % (NSETS, NSETS * nelem * 16 / 1e9),
                        "parallelism": "independent batches per GPU, no collective"},
-            "ms_per_step_median": per[len(per) // 2],
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                          "frac": achieved / peak, "peak_kind": peak_kind + " copy bandwidth",
                          "frac_of_nominal_8000": achieved / 8000.0,

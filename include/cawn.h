@@ -61,7 +61,16 @@ typedef enum cawn_status {
 
 enum {
     CAWN_FLAG_PRELUDE_CLAMP_SILU = 1u << 0, /* fused path: clamp conv output to +-50, then SiLU   */
-    CAWN_FLAG_RETENTION_DYNAMIC  = 1u << 1  /* gamma_t = sigmoid(gamma_logit[b,t,h] + freq_bias[k]) */
+    CAWN_FLAG_RETENTION_DYNAMIC  = 1u << 1, /* gamma_t = sigmoid(gamma_logit[b,t,h] + freq_bias[k]) */
+    CAWN_FLAG_INPUT_INDEPENDENT  = 1u << 2  /* forward: the caller vouches that `input`, gamma, theta
+                                               (and the conv weights) are not written by the call
+                                               made just before this one on the same stream.  The
+                                               kernels are launched so that a call may start while the
+                                               previous one drains (programmatic dependent launch);
+                                               with this flag the new call also fetches its input rows
+                                               during that overlap.  States, masks, workspaces and all
+                                               outputs are only touched once the previous call is
+                                               complete, with or without the flag.                    */
 };
 
 /* Operation selector of cawn_workspace_bytes(). */

@@ -26,6 +26,7 @@ CAWN_ERR_CARRY_TIMEOUT = 1
 
 CAWN_FLAG_PRELUDE_CLAMP_SILU = 1
 CAWN_FLAG_RETENTION_DYNAMIC = 2
+CAWN_FLAG_INPUT_INDEPENDENT = 4
 
 CAWN_OP_FWD, CAWN_OP_BWD_SAVED, CAWN_OP_BWD_PUSHES, CAWN_OP_STATE, CAWN_OP_FWD_HOST = range(5)
 CAWN_SAVED_STATES, CAWN_SAVED_PUSHES = 0, 1

@@ -76,7 +76,7 @@ int check_params(const cawn_params *p)
     if (p->B < 1 || p->L < 0 || p->H < 1 || p->F < 1) return CAWN_ERR_INVALID_ARG;
     if ((int64_t)p->H * p->F > (1 << 24)) return CAWN_ERR_INVALID_ARG;
     if (p->conv_k < 0) return CAWN_ERR_INVALID_ARG;
-    if (p->flags & ~(uint32_t)(CAWN_FLAG_PRELUDE_CLAMP_SILU | CAWN_FLAG_RETENTION_DYNAMIC))
+    if (p->flags & ~(uint32_t)(CAWN_FLAG_PRELUDE_CLAMP_SILU | CAWN_FLAG_RETENTION_DYNAMIC | CAWN_FLAG_INPUT_INDEPENDENT))
         return CAWN_ERR_INVALID_ARG;
     if (!(p->gate_eps >= 0.f)) return CAWN_ERR_INVALID_ARG;
     return CAWN_OK;
@@ -113,9 +113,20 @@ cudaError_t launch_scan_inst(const ScanParams &sp, cudaStream_t st)
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) configured[dev] = true;
     }
-    const dim3 grid((unsigned)sp.G, (unsigned)sp.B, (unsigned)sp.K);
-    cawn_scan_kernel<T, W, KIND, VEC, MINB, DYN><<<grid, W * 32, smem, st>>>(sp);
-    return cudaGetLastError();
+    // Launched with programmatic stream serialisation: when the launch before it on the stream
+    // is one of these kernels, this one may start occupying SMs while that one drains; the
+    // kernel itself waits for its predecessor before touching anything that one may have written.
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)sp.G, (unsigned)sp.B, (unsigned)sp.K);
+    cfg.blockDim = dim3(W * 32, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, cawn_scan_kernel<T, W, KIND, VEC, MINB, DYN>, sp);
 }
 template <int T, int W, int KIND, int MINB, bool DYN = false>
 cudaError_t launch_scan(const ScanParams &sp, cudaStream_t st)
@@ -321,6 +332,7 @@ int cawn_phase_accumulate_fwd(const cawn_params *params, const void *input,
         sp.conv_k = params->conv_k;
         sp.clamp_silu = (params->flags & CAWN_FLAG_PRELUDE_CLAMP_SILU) ? 1 : 0;
         sp.gate_tau = params->gate_tau;
+        sp.early_loads = (params->flags & CAWN_FLAG_INPUT_INDEPENDENT) ? 1 : 0;
         if (params->conv_k > 1) {
             sp.tail_in = state_in ? reinterpret_cast<const float *>(reinterpret_cast<const char *>(state_in) + tail_off) : nullptr;
             sp.tail_out = state_out ? reinterpret_cast<float *>(reinterpret_cast<char *>(state_out) + tail_off) : nullptr;
@@ -329,6 +341,7 @@ int cawn_phase_accumulate_fwd(const cawn_params *params, const void *input,
         return CAWN_OK;
     }
     sp.gamma_logit = gamma_logit; sp.freq_bias = freq_bias; sp.H = params->H; sp.F = params->F;
+    sp.early_loads = (params->flags & CAWN_FLAG_INPUT_INDEPENDENT) ? 1 : 0;
     if (launch_fwd(ts, sp, st, dyn) != cudaSuccess) return CAWN_ERR_CUDA;
     return CAWN_OK;
 }

@@ -85,6 +85,8 @@ struct ScanParams {
     int H, F;
     float *grad_logit;           // BWD: [B][L][H], zeroed before the launch (atomic adds)
     float *spart;                // BWD: per-tile partial sums of the logit gradient [B*K][C]
+    int early_loads;             // the input rows may be fetched before the preceding launch on the
+                                 // stream has finished (the caller vouches they are not its output)
 };
 
 // Shared memory of one CTA: the tile (two tiles in the backward: grad_y and P_{t-1}), then the
@@ -121,6 +123,11 @@ __device__ __forceinline__ void cp_async4(uint32_t dst, const void *src)
 {
     asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" :: "r"(dst), "l"(src) : "memory");
 }
+// Programmatic dependent launch: let the next launch on the stream start filling SMs as soon as
+// every CTA of this one is running, and wait for the previous launch (and its memory) to be
+// complete.  Both are no-ops for a launch made without the programmatic attribute.
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void grid_wait_previous() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 // Wait until at most n of this thread's most recent copy groups are still in flight (n <= 4).
@@ -196,6 +203,10 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
     // phase 3 only) is one more group behind them.
     constexpr int GR = T < 4 ? T : 4, NG = T / GR;
     static_assert(T % GR == 0 && NG <= 4, "copy groups");
+    // Unless the caller vouched for the input rows, nothing is read before the previous launch
+    // on the stream is complete.
+    const bool early = (KIND != KIND_BWD) && prm.early_loads != 0;
+    if (!early) grid_wait_previous();
     // Fused path: the hidden rows (floats) are staged in the upper part of the tile, behind
     // kHalo rows of history; phase 1 takes them into registers before the pushes overwrite them.
     float *const hs = reinterpret_cast<float *>(&sm.tile[0][0][0]) + (TILE * 128 - (TILE + kHalo) * 64);
@@ -216,7 +227,9 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
             r += C;
         }
         // history rows in front of the tile: earlier rows of h, or the carried tail before t = 0
+        // (the tail is the previous call's output: never before that call is complete)
         const int Kh = prm.conv_k - 1;
+        if (early) grid_wait_previous();
         if (w == 0) {
             const long long t0 = (long long)k * TILE;
 #pragma unroll
@@ -267,6 +280,8 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
         sm.sCoef[cl][2 * task] = re;
         sm.sCoef[cl][2 * task + 1] = im;
     }
+    // everything below touches what the previous launch may have written (workspace, states)
+    if (early && KIND != KIND_FUSED) grid_wait_previous();
     unsigned long long epoch0 = 0;
     unsigned arrived = 0;
     if (tid == 0) {
@@ -754,6 +769,7 @@ __global__ void __launch_bounds__(W * 32, MINB) cawn_scan_kernel(const ScanParam
     // (smaller k) always have smaller linear block indices
     const int g = blockIdx.x, b = blockIdx.y;
     const int k = blockIdx.z;                         // tile index along (logical) time
+    grid_launch_dependents();
     const bool full = ((long long)(k + 1) * TILE <= prm.L) && (g * 64 + 64 <= prm.C);
     if (full) scan_tile<T, W, KIND, VEC, DYN, true>(prm, sm, g, b, k);
     else      scan_tile<T, W, KIND, VEC, DYN, false>(prm, sm, g, b, k);
