@@ -142,6 +142,14 @@ __device__ __forceinline__ void cp_async_wait_pending(int n)
     }
 }
 
+// base + i * step in one instruction (step fits 32 bits: a row is at most 2^27 bytes)
+__device__ __forceinline__ const char *row_ptr(const char *base, int step, int i)
+{
+    long long r;
+    asm("mad.wide.s32 %0, %1, %2, %3;" : "=l"(r) : "r"(step), "r"(i), "l"((long long)base));
+    return reinterpret_cast<const char *>(r);
+}
+
 // Copy (asynchronously) or zero one row piece of this lane: two adjacent complex64 at byte
 // offset OFF from the thread's first piece (`dst` generic, `dst_s` the same in shared space).
 template <bool VEC, int OFF>
@@ -161,14 +169,14 @@ __device__ __forceinline__ void fetch_piece(float4 *dst, uint32_t dst_s, const c
 // global memory, 512 bytes apart in shared memory), committing one copy group per GR rows
 // (GR = 0: the caller commits).  valid(i) says whether row i exists.
 template <bool VEC, int T, int GR, int I = 0, typename F>
-__device__ __forceinline__ void fetch_rows(float4 *dst, uint32_t dst_s, const char *src, long long step,
+__device__ __forceinline__ void fetch_rows(float4 *dst, uint32_t dst_s, const char *src, int step,
                                            bool vA, bool vB, F valid)
 {
     if constexpr (I < T) {
         const bool row = valid(I);
-        fetch_piece<VEC, I * 512>(dst, dst_s, src, row && vA, row && vB);
+        fetch_piece<VEC, I * 512>(dst, dst_s, row_ptr(src, step, I), row && vA, row && vB);
         if constexpr (GR > 0 && (I + 1) % GR == 0) cp_async_commit();
-        fetch_rows<VEC, T, GR, I + 1>(dst, dst_s, src + step, step, vA, vB, valid);
+        fetch_rows<VEC, T, GR, I + 1>(dst, dst_s, src, step, vA, vB, valid);
     }
 }
 
@@ -193,7 +201,7 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
     }
     // logical step s <-> physical row t: forward t = s, reverse t = L-1-s
     const long long t_first = REV ? (L - 1 - s0) : s0;
-    const long long rowbytes = (REV ? -(long long)C : (long long)C) * 8;
+    const int rowbytes = (REV ? -C : C) * 8;
     const long long e0 = ((long long)b * L + t_first) * C + c0;    // only used when nvalid > 0
     float4 *const xs = &sm.tile[0][w * T][lane];                   // this thread's pieces, 32 float4 apart
 
@@ -201,7 +209,7 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
     // The rows go out as NG copy groups of GR rows each, so that phase 1 can start on the first
     // rows while the later ones are still in flight.  The backward's second tile (needed in
     // phase 3 only) is one more group behind them.
-    constexpr int GR = T < 4 ? T : 4, NG = T / GR;
+    constexpr int GR = T < 4 ? T : (T > 16 ? T / 4 : 4), NG = T / GR;
     static_assert(T % GR == 0 && NG <= 4, "copy groups");
     // Unless the caller vouched for the input rows, nothing is read before the previous launch
     // on the stream is complete.
@@ -615,7 +623,7 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
             else P = cfma2(aT, P, sm.sE[i][lane]);
         }
 
-        char *r = reinterpret_cast<char *>(prm.out) + e0 * 8;
+        char *const rbase = reinterpret_cast<char *>(prm.out) + e0 * 8;
         const float cl = prm.clampv;
         // DYN: factor of the step into row i (forward: the row's own; backward: the factor of
         // the row processed before it), and the running sum of the logit gradient
@@ -632,6 +640,7 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
                     P = cfma2(a, P, xs[i * 32]);
                 }
                 const float4 o = clamped ? clamp4(P, cl) : P;
+                char *r = const_cast<char *>(row_ptr(rbase, rowbytes, i));
                 if (VEC) {
                     if (vA) __stcs(reinterpret_cast<float4 *>(r), o);
                 } else {
@@ -676,7 +685,6 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
                     }
                 }
             }
-            r += rowbytes;
         };
         if (cl > 0.f) {
 #pragma unroll
