@@ -1,0 +1,154 @@
+"""Device-time measurements of the other benchmark configs (bench.py times config 1 only).
+
+    python -m paper_2604_04250_b200.bench_configs [--steps K] [--warmup W]
+
+Prints one JSON line per workload: config 3 (backward, saved states), config 4 (fused mixing
+path), config 2 (chunked prefill, a window of 4096-token calls with state passing), config 1 with
+the mask emitted, and config 1 with time-varying retention.  Inputs are the seeded synthetic
+arrays of ``inputs.py``, resident on the device; steps rotate over several buffer sets so that
+no step finds its inputs in L2; K steps are timed between two CUDA events.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+
+import numpy as np
+
+
+def _peak():
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    try:
+        with open(os.path.join(root, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+def _time(step, steps, warmup):
+    import torch
+    st = torch.cuda.current_stream()
+    for i in range(warmup):
+        step(i)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(st)
+    for i in range(steps):
+        step(warmup + i)
+    e1.record(st)
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / steps
+
+
+def _report(name, tokens, bytes_per_step, ms, launches, extra=None):
+    peak, kind = _peak()
+    gbs = bytes_per_step / (ms * 1e-3) / 1e9
+    line = {"workload": name, "ms_per_step": ms, "Mtokens_per_s": tokens / (ms * 1e-3) / 1e6,
+            "algorithmic_GBps": gbs, "frac_of_%s_copy_peak" % kind: gbs / peak,
+            "frac_of_nominal_8000": gbs / 8000.0, "launches_per_step": launches}
+    if extra:
+        line.update(extra)
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    args = ap.parse_args()
+    import torch
+    from . import binding as cb, inputs
+    cb.lib()
+    torch.cuda.set_device(0)
+    dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
+    IND = cb.CAWN_FLAG_INPUT_INDEPENDENT
+
+    # ---- config 1 with the gate mask emitted, and with time-varying retention -----------------
+    cfg = inputs.CONFIGS[1]
+    B, L, C = cfg.B, cfg.L, cfg.C
+    d = inputs.scan_inputs(B, L, C, cfg.seed, cfg.gamma_lo, cfg.gamma_hi)
+    g, t, p0 = dev(d["gamma"]), dev(d["theta"]), dev(d["p"])
+    NS = 6
+    ps = [torch.roll(p0, 17 * i, 1).contiguous() for i in range(NS)]
+    ys = [torch.empty_like(p0) for _ in range(NS)]
+    masks = [torch.zeros((B, L, C // 32), dtype=torch.int32, device="cuda") for _ in range(NS)]
+    prm = cb.make_params(B, L, cfg.H, cfg.F, gate_eps=cfg.gate_eps, flags=IND)
+    ws = cb.new_workspace(prm, cb.CAWN_OP_FWD)
+    ms = _time(lambda i: cb.cawn_phase_accumulate_fwd(prm, ps[i % NS], g, t, ys[i % NS], ws, gate_mask=masks[i % NS]),
+               args.steps, args.warmup)
+    _report("cfg1_train_fwd+mask", B * L, B * L * C * (16 + 0.125), ms, 1)
+    dd = inputs.dynamic_retention_inputs(B, L, cfg.H, cfg.F, 7)
+    gl, fb = dev(dd["gamma_logit"]), dev(dd["freq_bias"])
+    prm_d = cb.make_params(B, L, cfg.H, cfg.F, gate_eps=cfg.gate_eps, flags=IND | cb.CAWN_FLAG_RETENTION_DYNAMIC)
+    ms = _time(lambda i: cb.cawn_phase_accumulate_fwd(prm_d, ps[i % NS], None, t, ys[i % NS], ws, gamma_logit=gl, freq_bias=fb),
+               args.steps, args.warmup)
+    _report("cfg1_train_fwd_dynamic_retention", B * L, B * L * (C * 16 + cfg.H * 4), ms, 1)
+    assert cb.cawn_poll_status(ws) == 0
+    del ps, ys, masks
+
+    # ---- config 3: backward with saved states ---------------------------------------------------
+    cfg = inputs.CONFIGS[3]
+    B, L, C = cfg.B, cfg.L, cfg.C
+    d = inputs.config_inputs(cfg)
+    g, t = dev(d["gamma"]), dev(d["theta"])
+    prm = cb.make_params(B, L, cfg.H, cfg.F, gate_eps=cfg.gate_eps)
+    NS = 3
+    P = torch.empty((B, L, C), dtype=torch.complex64, device="cuda")
+    wf = cb.new_workspace(prm, cb.CAWN_OP_FWD)
+    cb.cawn_phase_accumulate_fwd(prm, dev(d["p"]), g, t, P, wf)
+    Ps = [P.clone() for _ in range(NS)]
+    gys = [dev(d["grad_y"]) for _ in range(NS)]
+    gps = [torch.empty_like(P) for _ in range(NS)]
+    gg, gt = torch.empty(C, device="cuda"), torch.empty(C, device="cuda")
+    gsi = torch.empty((B, C), dtype=torch.complex64, device="cuda")
+    wb = cb.new_workspace(prm, cb.CAWN_OP_BWD_SAVED)
+    ms = _time(lambda i: cb.cawn_phase_accumulate_bwd(prm, Ps[i % NS], cb.CAWN_SAVED_STATES, g, t, gys[i % NS], gps[i % NS],
+                                                      wb, grad_gamma=gg, grad_theta=gt, grad_state_in=gsi),
+               args.steps, args.warmup)
+    assert cb.cawn_poll_status(wb) == 0
+    _report("cfg3_bwd", B * L, B * L * C * 24, ms, 2, {"note": "reads grad_y and saved P, writes grad_p; plus the finalize kernel"})
+    del Ps, gys, gps, P
+
+    # ---- config 4: fused mixing path -------------------------------------------------------------
+    cfg = inputs.CONFIGS[4]
+    B, L, C = cfg.B, cfg.L, cfg.C
+    d = inputs.config_inputs(cfg)
+    g, t, w = dev(d["gamma"]), dev(d["theta"]), dev(d["conv_w"])
+    prm = cb.make_params(B, L, cfg.H, cfg.F, gate_eps=cfg.gate_eps, gate_tau=float(inputs.gate_tau(cfg.gate_eps)),
+                         conv_k=cfg.conv_k, flags=IND)
+    NS = 2
+    hs = [dev(d["h"]) for _ in range(NS)]
+    ys = [torch.empty((B, L, C), dtype=torch.complex64, device="cuda") for _ in range(NS)]
+    ws = cb.new_workspace(prm, cb.CAWN_OP_FWD)
+    ms = _time(lambda i: cb.cawn_phase_accumulate_fwd(prm, hs[i % NS], g, t, ys[i % NS], ws, conv_w=w),
+               max(args.steps // 2, 5), args.warmup)
+    assert cb.cawn_poll_status(ws) == 0
+    _report("cfg4_fused", B * L, B * L * C * 12, ms, 1)
+    del hs, ys
+
+    # ---- config 2: chunked prefill, 64 calls of 4096 tokens with the state carried ---------------
+    cfg = inputs.CONFIGS[2]
+    C, n = cfg.C, cfg.chunk
+    stream = inputs.prefill_stream(cfg, total=16 * n)
+    gamma, theta = next(stream)
+    g, t = dev(gamma), dev(theta)
+    chunks = [dev(p) for p in stream]                     # 16 distinct chunks (805 MB), cycled
+    ys = [torch.empty_like(chunks[0]) for _ in range(4)]
+    state = torch.zeros((cfg.B, C), dtype=torch.complex64, device="cuda")
+    prm = cb.make_params(cfg.B, n, cfg.H, cfg.F, gate_eps=cfg.gate_eps, flags=IND)
+    ws = cb.new_workspace(prm, cb.CAWN_OP_FWD)
+    ncalls = 64
+
+    def prefill(i):
+        for j in range(ncalls):
+            cb.cawn_phase_accumulate_fwd(prm, chunks[j % 16], g, t, ys[j % 4], ws, state_in=state, state_out=state)
+    ms = _time(prefill, max(args.steps // 10, 3), 2)
+    assert cb.cawn_poll_status(ws) == 0
+    _report("cfg2_chunked_prefill", ncalls * n, ncalls * n * C * 16, ms, ncalls,
+            {"us_per_4096_token_call": ms * 1e3 / ncalls, "note": "one launch per chunk, state carried on the device"})
+
+
+if __name__ == "__main__":
+    sys.exit(main())
