@@ -29,8 +29,10 @@ UNIT = "Mtokens/s"
 NSETS = 6                      # rotating buffer sets: 6 x 201 MB = 1.2 GB >> 126 MB of L2
 BYTES_PER_ELEMENT = 16         # algorithmic: read one complex64 push, write one complex64 output
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the scan kernel on this
-# workload, from the ncu capture summarised in profiles/ (None until captured).
-NCU_DRAM_BYTES_PER_LAUNCH = None
+# workload, from the ncu capture summarised in profiles/cawn_scan_fwd_cfg1_ncu.md: 101.5 MB read
+# + 47.5 MB written while an isolated launch runs (the rest of its 100.7 MB of output is still
+# dirty in L2 when it ends).  Set to None whenever the kernel changes after the capture.
+NCU_DRAM_BYTES_PER_LAUNCH = 149061888
 
 
 def workload():
@@ -144,6 +146,26 @@ def run_reference(args):
     }))
 
 
+def rank_seed(cfg_seed, rank):
+    """Every rank draws its own batch shard: same recipe, rank-specific seed."""
+    return cfg_seed + 1000 * rank
+
+
+def reduce_max(values, world, device):
+    """Max over ranks of a few per-rank timings (the slowest rank defines the step time)."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t.cpu()]
+
+
+def whole_job_value(world, tokens_per_rank, ms_per_step):
+    """Mtokens/s of all ranks together (weak scaling: every rank processes its own batch shard)."""
+    return world * tokens_per_rank / (ms_per_step * 1e-3) / 1e6
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -163,7 +185,7 @@ def run_ours(args):
     nelem = tokens * C
     # every step reads a buffer set that no earlier step writes: the calls may overlap their tails
     prm = cb.make_params(B, L, cfg.H, cfg.F, gate_eps=cfg.gate_eps, flags=cb.CAWN_FLAG_INPUT_INDEPENDENT)
-    d = inputs.scan_inputs(B, L, C, cfg.seed + 1000 * rank, cfg.gamma_lo, cfg.gamma_hi)
+    d = inputs.scan_inputs(B, L, C, rank_seed(cfg.seed, rank), cfg.gamma_lo, cfg.gamma_hi)
     gamma = torch.from_numpy(d["gamma"]).cuda()
     theta = torch.from_numpy(d["theta"]).cuda()
     p0 = torch.from_numpy(d["p"]).cuda()
@@ -222,10 +244,7 @@ def run_ours(args):
     e2e_ms = e0.elapsed_time(e1) / e2e_steps
     clocks = sampler.stop() if rank == 0 else None
 
-    times = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    total_ms, e2e_ms = (float(x) for x in times.cpu())
+    total_ms, e2e_ms = reduce_max([total_ms, e2e_ms], world, "cuda")
     ms_per_step = total_ms / args.steps
 
     if rank == 0:
@@ -239,7 +258,7 @@ def run_ours(args):
                    "sample": "%d full passes of the same workload (B=%d L=%d C=%d) in %.1f s, one thread"
                              % (passes, B, L, C, dt)}
         line = {
-            "metric": METRIC, "value": world * tokens / (ms_per_step * 1e-3) / 1e6, "unit": UNIT,
+            "metric": METRIC, "value": whole_job_value(world, tokens, ms_per_step), "unit": UNIT,
             "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
             "data": "synthetic",
@@ -251,10 +270,10 @@ def run_ours(args):
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                          "frac": achieved / peak, "peak_kind": peak_kind + " copy bandwidth",
                          "frac_of_nominal_8000": achieved / 8000.0,
-                         "kernel": "cawn_scan_kernel<16,8,FWD>", "kernel_ms": kernel_ms,
+                         "kernel": "cawn_scan_kernel<16,8,KIND_FWD,VEC,3>", "kernel_ms": kernel_ms,
                          "algorithmic_bytes_per_launch": nelem * BYTES_PER_ELEMENT,
                          "traffic": NCU_DRAM_BYTES_PER_LAUNCH},
-            "e2e": {"value": world * tokens / (e2e_ms * 1e-3) / 1e6, "unit": UNIT,
+            "e2e": {"value": whole_job_value(world, tokens, e2e_ms), "unit": UNIT,
                     "h2d_bytes_per_step": nelem * 8 + 2 * C * 4, "d2h_bytes_per_step": nelem * 8 + B * C * 8,
                     "ms_per_step": e2e_ms, "api": "cawn_phase_accumulate_fwd_host (pinned host buffers)"},
             "gpu_launches": args.steps,

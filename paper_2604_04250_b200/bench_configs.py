@@ -57,7 +57,11 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--only", default="", help="comma-separated subset of: mask,dynamic,cfg3,cfg4,cfg2")
+    ap.add_argument("--cfg4-batch", type=int, default=0, help="batch rows of the config-4 run (0: the config's 16)")
     args = ap.parse_args()
+    only = set(x for x in args.only.split(",") if x)
+    want = lambda name: not only or name in only
     import torch
     from . import binding as cb, inputs
     cb.lib()
@@ -76,18 +80,30 @@ def main():
     masks = [torch.zeros((B, L, C // 32), dtype=torch.int32, device="cuda") for _ in range(NS)]
     prm = cb.make_params(B, L, cfg.H, cfg.F, gate_eps=cfg.gate_eps, flags=IND)
     ws = cb.new_workspace(prm, cb.CAWN_OP_FWD)
-    ms = _time(lambda i: cb.cawn_phase_accumulate_fwd(prm, ps[i % NS], g, t, ys[i % NS], ws, gate_mask=masks[i % NS]),
-               args.steps, args.warmup)
-    _report("cfg1_train_fwd+mask", B * L, B * L * C * (16 + 0.125), ms, 1)
-    dd = inputs.dynamic_retention_inputs(B, L, cfg.H, cfg.F, 7)
-    gl, fb = dev(dd["gamma_logit"]), dev(dd["freq_bias"])
-    prm_d = cb.make_params(B, L, cfg.H, cfg.F, gate_eps=cfg.gate_eps, flags=IND | cb.CAWN_FLAG_RETENTION_DYNAMIC)
-    ms = _time(lambda i: cb.cawn_phase_accumulate_fwd(prm_d, ps[i % NS], None, t, ys[i % NS], ws, gamma_logit=gl, freq_bias=fb),
-               args.steps, args.warmup)
-    _report("cfg1_train_fwd_dynamic_retention", B * L, B * L * (C * 16 + cfg.H * 4), ms, 1)
+    if want("mask"):
+        ms = _time(lambda i: cb.cawn_phase_accumulate_fwd(prm, ps[i % NS], g, t, ys[i % NS], ws, gate_mask=masks[i % NS]),
+                   args.steps, args.warmup)
+        _report("cfg1_train_fwd+mask", B * L, B * L * C * (16 + 0.125), ms, 1)
+    if want("dynamic"):
+        dd = inputs.dynamic_retention_inputs(B, L, cfg.H, cfg.F, 7)
+        gl, fb = dev(dd["gamma_logit"]), dev(dd["freq_bias"])
+        prm_d = cb.make_params(B, L, cfg.H, cfg.F, gate_eps=cfg.gate_eps, flags=IND | cb.CAWN_FLAG_RETENTION_DYNAMIC)
+        ms = _time(lambda i: cb.cawn_phase_accumulate_fwd(prm_d, ps[i % NS], None, t, ys[i % NS], ws, gamma_logit=gl, freq_bias=fb),
+                   args.steps, args.warmup)
+        _report("cfg1_train_fwd_dynamic_retention", B * L, B * L * (C * 16 + cfg.H * 4), ms, 1)
     assert cb.cawn_poll_status(ws) == 0
     del ps, ys, masks
 
+    if want("cfg3"):
+        _cfg3(args, cb, inputs, dev)
+    if want("cfg4"):
+        _cfg4(args, cb, inputs, dev, IND)
+    if want("cfg2"):
+        _cfg2(args, cb, inputs, dev, IND)
+
+
+def _cfg3(args, cb, inputs, dev):
+    import torch
     # ---- config 3: backward with saved states ---------------------------------------------------
     cfg = inputs.CONFIGS[3]
     B, L, C = cfg.B, cfg.L, cfg.C
@@ -109,12 +125,14 @@ def main():
                args.steps, args.warmup)
     assert cb.cawn_poll_status(wb) == 0
     _report("cfg3_bwd", B * L, B * L * C * 24, ms, 2, {"note": "reads grad_y and saved P, writes grad_p; plus the finalize kernel"})
-    del Ps, gys, gps, P
 
+
+def _cfg4(args, cb, inputs, dev, IND):
+    import torch
     # ---- config 4: fused mixing path -------------------------------------------------------------
     cfg = inputs.CONFIGS[4]
-    B, L, C = cfg.B, cfg.L, cfg.C
-    d = inputs.config_inputs(cfg)
+    B, L, C = (args.cfg4_batch or cfg.B), cfg.L, cfg.C
+    d = inputs.fused_inputs(B, L, C, cfg.seed, cfg.conv_k, cfg.gamma_lo, cfg.gamma_hi)
     g, t, w = dev(d["gamma"]), dev(d["theta"]), dev(d["conv_w"])
     prm = cb.make_params(B, L, cfg.H, cfg.F, gate_eps=cfg.gate_eps, gate_tau=float(inputs.gate_tau(cfg.gate_eps)),
                          conv_k=cfg.conv_k, flags=IND)
@@ -125,9 +143,11 @@ def main():
     ms = _time(lambda i: cb.cawn_phase_accumulate_fwd(prm, hs[i % NS], g, t, ys[i % NS], ws, conv_w=w),
                max(args.steps // 2, 5), args.warmup)
     assert cb.cawn_poll_status(ws) == 0
-    _report("cfg4_fused", B * L, B * L * C * 12, ms, 1)
-    del hs, ys
+    _report("cfg4_fused" if B == cfg.B else "cfg4_fused_B%d" % B, B * L, B * L * C * 12, ms, 1)
 
+
+def _cfg2(args, cb, inputs, dev, IND):
+    import torch
     # ---- config 2: chunked prefill, 64 calls of 4096 tokens with the state carried ---------------
     cfg = inputs.CONFIGS[2]
     C, n = cfg.C, cfg.chunk
