@@ -135,6 +135,32 @@ cudaError_t launch_scan(const ScanParams &sp, cudaStream_t st)
                          : launch_scan_inst<T, W, KIND, false, MINB, DYN>(sp, st);
 }
 
+// First-wave stagger of the static forward scan: about two thirds of the time one SM's share of
+// HBM bandwidth needs for a tile's input and output.  Device numbers are read once per device.
+void set_stagger(ScanParams &sp, TileShape ts)
+{
+    static int sms[64] = {}, cycles_per_byte_q20[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return;
+    if (sms[dev] == 0) {
+        int n = 0, mem_khz = 0, bus_bits = 0, sm_khz = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&mem_khz, cudaDevAttrMemoryClockRate, dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&bus_bits, cudaDevAttrGlobalMemoryBusWidth, dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&sm_khz, cudaDevAttrClockRate, dev) != cudaSuccess ||
+            n <= 0 || mem_khz <= 0 || bus_bits <= 0 || sm_khz <= 0)
+            return;
+        // achievable bandwidth taken as 0.8 of 2 x memory clock x bus width, split over the SMs
+        const double bytes_per_s = 0.8 * 2.0 * (double)mem_khz * 1e3 * (double)bus_bits / 8.0 / (double)n;
+        cycles_per_byte_q20[dev] = (int)((double)sm_khz * 1e3 / bytes_per_s * 1048576.0);
+        sms[dev] = n;
+    }
+    const long long tile_bytes = (long long)ts.T * ts.W * 64 * 16;     // input + output of one tile
+    sp.stagger_cycles = (int)((tile_bytes * cycles_per_byte_q20[dev] * 2 / 3) >> 20);
+    sp.stagger_group = sms[dev];
+    sp.stagger_slots = 3;
+}
+
 inline cudaError_t launch_fwd(TileShape ts, const ScanParams &sp, cudaStream_t st, bool dyn = false)
 {
     if (dyn) {
@@ -342,6 +368,7 @@ int cawn_phase_accumulate_fwd(const cawn_params *params, const void *input,
     }
     sp.gamma_logit = gamma_logit; sp.freq_bias = freq_bias; sp.H = params->H; sp.F = params->F;
     sp.early_loads = (params->flags & CAWN_FLAG_INPUT_INDEPENDENT) ? 1 : 0;
+    if (!dyn && ts.T == 16) set_stagger(sp, ts);
     if (launch_fwd(ts, sp, st, dyn) != cudaSuccess) return CAWN_ERR_CUDA;
     return CAWN_OK;
 }

@@ -85,6 +85,11 @@ struct ScanParams {
     int H, F;
     float *grad_logit;           // BWD: [B][L][H], zeroed before the launch (atomic adds)
     float *spart;                // BWD: per-tile partial sums of the logit gradient [B*K][C]
+    // First-wave stagger: the CTAs that land in the 2nd, 3rd, ... resident slot of an SM (linear
+    // block index / stagger_group) start their copies stagger_cycles, 2 stagger_cycles, ... late,
+    // so that the CTAs sharing an SM run out of phase and their load, arithmetic and store
+    // phases overlap instead of alternating.  0 = off.
+    int stagger_cycles, stagger_group, stagger_slots;
     int early_loads;             // the input rows may be fetched before the preceding launch on the
                                  // stream has finished (the caller vouches they are not its output)
 };
@@ -213,6 +218,17 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
     static_assert(T % GR == 0 && NG <= 4, "copy groups");
     // Unless the caller vouched for the input rows, nothing is read before the previous launch
     // on the stream is complete.
+    if (prm.stagger_cycles > 0) {
+        const unsigned lin = (blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x;
+        const unsigned slot = lin / (unsigned)prm.stagger_group;
+        if (slot >= 1u && slot < (unsigned)prm.stagger_slots) {
+            if (tid == 0) {
+                const long long t0 = clock64(), target = (long long)slot * prm.stagger_cycles;
+                for (int it = 0; it < 4096 && clock64() - t0 < target; ++it) __nanosleep(64);
+            }
+            __syncthreads();
+        }
+    }
     const bool early = (KIND != KIND_BWD) && prm.early_loads != 0;
     if (!early) grid_wait_previous();
     // Fused path: the hidden rows (floats) are staged in the upper part of the tile, behind
@@ -399,42 +415,47 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
         const bool want_mask = prm.mask != nullptr;
         uint32_t *mrow = prm.mask + ((long long)b * L + s0) * prm.MW + g * 2;
         const bool second_word = g * 2 + 1 < prm.MW;
-        auto phasor = [&](float u, bool valid, float &zr, float &zi) -> bool {
-            float x = u;
+        // All of it runs two channels wide on packed fp32 pairs (fma.rn.f32x2 and friends): a
+        // lane's hidden values already come as (channel, channel+1) pairs, and the pushes are
+        // kept in shared memory as (re, re, im, im) so that the scan stays two wide as well.
+        float2 w2[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) w2[j] = make_float2(wA[j], wB[j]);
+        const float2 b2 = make_float2(bA, bB);
+        const float2 ar2 = make_float2(a.x, a.z), ai2 = make_float2(a.y, a.w), nai2 = make_float2(-a.y, -a.w);
+        const float2 one2 = make_float2(1.f, 1.f);
+        float2 er2 = make_float2(0.f, 0.f), ei2 = er2;
+#pragma unroll
+        for (int i = 0; i < T; ++i) {
+            float2 u = b2;
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if (j >= 4 - Kc) u = __ffma2_rn(w2[j], hv[i + j], u);     // fmaf per channel, tap order
+            float2 x = u;
             if (act) {
-                x = fminf(fmaxf(x, -50.f), 50.f);
-                x = __fdividef(x, 1.f + __expf(-x));
+                x.x = fminf(fmaxf(x.x, -50.f), 50.f); x.y = fminf(fmaxf(x.y, -50.f), 50.f);
+                x.x = __fdividef(x.x, 1.f + __expf(-x.x)); x.y = __fdividef(x.y, 1.f + __expf(-x.y));
             }
             // one exponential serves both maps: with q = e^-x, sigmoid = 1/(1+q) and
             // tanh = (1-q^2)/(1+q^2); |x| is capped where both have long saturated in fp32
-            const float xc = fminf(fmaxf(x, -25.f), 25.f);
-            const float q = __expf(-xc), q2 = q * q;
-            const float rcp = __fdividef(1.f, (1.f + q) * (1.f + q2));
-            const float m = (1.f + q2) * rcp;
-            const float th = (1.f - q2) * (1.f + q) * rcp;
-            float sn, cs;
-            __sincosf(3.14159265358979f * th, &sn, &cs);
+            const float2 xc = make_float2(fminf(fmaxf(x.x, -25.f), 25.f), fminf(fmaxf(x.y, -25.f), 25.f));
+            const float2 q = make_float2(__expf(-xc.x), __expf(-xc.y));
+            const float2 q2 = __fmul2_rn(q, q);
+            const float2 p1 = __fadd2_rn(q, one2), p2 = __fadd2_rn(q2, one2);
+            const float2 den = __fmul2_rn(p1, p2);
+            const float2 rcp = make_float2(__fdividef(1.f, den.x), __fdividef(1.f, den.y));
+            float2 m = __fmul2_rn(p2, rcp);
+            const float2 n1 = __ffma2_rn(q, make_float2(-q.x, -q.y), one2);
+            const float2 ang = __fmul2_rn(__fmul2_rn(__fmul2_rn(n1, p1), rcp), make_float2(3.14159265358979f, 3.14159265358979f));
+            float2 cs, sn;
+            __sincosf(ang.x, &sn.x, &cs.x);
+            __sincosf(ang.y, &sn.y, &cs.y);
             // with clamp + SiLU the magnitude never falls below 0.43, and the host only admits
             // thresholds under that: every gate is open
-            const bool open = valid && (act || u >= tau);
-            zr = open ? m * cs : 0.f;
-            zi = open ? m * sn : 0.f;
-            return open;
-        };
-#pragma unroll
-        for (int i = 0; i < T; ++i) {
-            float uA = bA, uB = bB;
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                if (j >= 4 - Kc) {
-                    uA = fmaf(wA[j], hv[i + j].x, uA);
-                    uB = fmaf(wB[j], hv[i + j].y, uB);
-                }
-            }
-            float4 v;
-            const bool oA = phasor(uA, vA, v.x, v.y);
-            const bool oB = phasor(uB, vB, v.z, v.w);
-            xs[i * 32] = v;
+            const bool oA = vA && (act || u.x >= tau), oB = vB && (act || u.y >= tau);
+            m.x = oA ? m.x : 0.f; m.y = oB ? m.y : 0.f;
+            const float2 zr = __fmul2_rn(m, cs), zi = __fmul2_rn(m, sn);
+            xs[i * 32] = make_float4(zr.x, zr.y, zi.x, zi.y);            // (re, re, im, im)
             if (want_mask) {
                 const unsigned bits = ((oA ? 1u : 0u) | (oB ? 2u : 0u)) << (2 * (lane & 15));
                 const unsigned w0 = __reduce_or_sync(0xffffffffu, lane < 16 ? bits : 0u);
@@ -445,8 +466,13 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
                 }
                 mrow += prm.MW;
             }
-            if (FULL || i < nvalid) e = cfma2(a, e, v);
+            if (FULL || i < nvalid) {
+                const float2 nr = __ffma2_rn(ar2, er2, __ffma2_rn(nai2, ei2, zr));
+                const float2 ni = __ffma2_rn(ar2, ei2, __ffma2_rn(ai2, er2, zi));
+                er2 = nr; ei2 = ni;
+            }
         }
+        e = make_float4(er2.x, ei2.x, er2.y, ei2.y);
     } else if constexpr (KIND == KIND_FWD) {
         // |p| >= eps decided as re^2 + im^2 >= eps^2 in double: both squares are exact there
         // and the sum rounds once, so the decision is reproducible bit for bit.  The fp32 sum
@@ -686,7 +712,31 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
                 }
             }
         };
-        if (cl > 0.f) {
+        if constexpr (KIND == KIND_FUSED) {
+            // the pushes sit in shared memory as (re, re, im, im): the recurrence runs two wide
+            const float2 ar2 = make_float2(a.x, a.z), ai2 = make_float2(a.y, a.w), nai2 = make_float2(-a.y, -a.w);
+            float2 Pr = make_float2(P.x, P.z), Pi = make_float2(P.y, P.w);
+#pragma unroll
+            for (int i = 0; i < T; ++i) {
+                if (FULL || i < nvalid) {
+                    const float4 z = xs[i * 32];
+                    const float2 nr = __ffma2_rn(ar2, Pr, __ffma2_rn(nai2, Pi, make_float2(z.x, z.y)));
+                    const float2 ni = __ffma2_rn(ar2, Pi, __ffma2_rn(ai2, Pr, make_float2(z.z, z.w)));
+                    Pr = nr; Pi = ni;
+                    float4 o = make_float4(Pr.x, Pi.x, Pr.y, Pi.y);
+                    if (cl > 0.f) o = clamp4(o, cl);
+                    char *r = const_cast<char *>(row_ptr(rbase, rowbytes, i));
+                    if (VEC) {
+                        if (vA) __stcs(reinterpret_cast<float4 *>(r), o);
+                    } else {
+                        float2 *r2 = reinterpret_cast<float2 *>(r);
+                        if (vA) __stcs(r2, make_float2(o.x, o.y));
+                        if (vB) __stcs(r2 + 1, make_float2(o.z, o.w));
+                    }
+                }
+            }
+            P = make_float4(Pr.x, Pi.x, Pr.y, Pi.y);
+        } else if (cl > 0.f) {
 #pragma unroll
             for (int i = 0; i < T; ++i) step_row(i, true);
         } else {
