@@ -29,10 +29,10 @@ UNIT = "Mtokens/s"
 NSETS = 6                      # rotating buffer sets: 6 x 201 MB = 1.2 GB >> 126 MB of L2
 BYTES_PER_ELEMENT = 16         # algorithmic: read one complex64 push, write one complex64 output
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the scan kernel on this
-# workload, from the ncu capture summarised in profiles/cawn_scan_fwd_cfg1_ncu.md: 101.5 MB read
-# + 47.5 MB written while an isolated launch runs (the rest of its 100.7 MB of output is still
+# workload, from the ncu capture summarised in profiles/cawn_scan_fwd_cfg1_ncu.md: 101.4 MB read
+# + 47.4 MB written while an isolated launch runs (the rest of its 100.7 MB of output is still
 # dirty in L2 when it ends).  Set to None whenever the kernel changes after the capture.
-NCU_DRAM_BYTES_PER_LAUNCH = 149061888
+NCU_DRAM_BYTES_PER_LAUNCH = 148722688
 
 
 def workload():
