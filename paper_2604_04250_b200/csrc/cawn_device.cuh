@@ -26,10 +26,6 @@ enum : unsigned { REC_AGGREGATE = 1u, REC_PREFIX = 2u, REC_POISON = 3u };
 
 // ---------------------------------------------------------------------------------------
 // Every lane works on two adjacent channels at once; a float4 holds (re0, im0, re1, im1).
-__device__ __forceinline__ float2 cmul(float2 a, float2 b)
-{
-    return make_float2(fmaf(a.x, b.x, -a.y * b.y), fmaf(a.x, b.y, a.y * b.x));
-}
 // a * b + c on both channels of a pair
 __device__ __forceinline__ float4 cfma2(float4 a, float4 b, float4 c)
 {
@@ -55,19 +51,6 @@ __device__ __forceinline__ float4 clamp4(float4 v, float c)
     return make_float4(clampf(v.x, c), clampf(v.y, c), clampf(v.z, c), clampf(v.w, c));
 }
 __device__ __forceinline__ float4 zero4() { return make_float4(0.f, 0.f, 0.f, 0.f); }
-
-// Integer power of a complex double by square-and-multiply (N is a compile-time constant).
-template <int N>
-__device__ __forceinline__ void cpow_int(double ar, double ai, double &rr, double &ri)
-{
-    double br = ar, bi = ai;
-    rr = 1.0; ri = 0.0;
-#pragma unroll
-    for (int n = N; n > 0; n >>= 1) {
-        if (n & 1) { const double t = rr * br - ri * bi; ri = rr * bi + ri * br; rr = t; }
-        const double t = br * br - bi * bi; bi = 2.0 * br * bi; br = t;
-    }
-}
 
 // ---------------------------------------------------------------------------------------
 // Carry records: {re, im, tag} in one aligned 16-byte word, written and read with single
