@@ -63,7 +63,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
-                 "--format=csv,noheader,nounits", "-lms", "100"],
+                 "--format=csv,noheader,nounits", "-lms", "20"],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except Exception:
             self.proc = None
@@ -208,9 +208,13 @@ def run_ours(args):
     for i in range(args.warmup):
         step(i)
     barrier()
+    # The timed region lasts a few milliseconds, nvidia-smi samples every 20 ms: the clocks are
+    # sampled over the K timed steps plus the same steps repeated (untimed) for about half a second
+    # right after them, so that the samples describe the GPU under this very load.
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
+        time.sleep(0.05)
     # two events bracket the K steps: an event between two launches would make each launch wait for
     # the one before to drain completely, which back-to-back calls on a stream do not do
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -220,6 +224,12 @@ def run_ours(args):
     ev1.record(stream)
     barrier()
     total_ms = ev0.elapsed_time(ev1)
+    t_load = time.perf_counter()
+    while time.perf_counter() - t_load < 0.5:
+        for i in range(50):
+            step(i)
+        torch.cuda.synchronize()
+    clocks_now = sampler.stop() if rank == 0 else None
     status = cb.cawn_poll_status(ws)
     if status != 0:
         raise RuntimeError("device status: " + cb.status_string(status))
@@ -242,7 +252,6 @@ def run_ours(args):
     e1.record(stream)
     barrier()
     e2e_ms = e0.elapsed_time(e1) / e2e_steps
-    clocks = sampler.stop() if rank == 0 else None
 
     total_ms, e2e_ms = reduce_max([total_ms, e2e_ms], world, "cuda")
     ms_per_step = total_ms / args.steps
@@ -277,7 +286,7 @@ def run_ours(args):
                     "h2d_bytes_per_step": nelem * 8 + 2 * C * 4, "d2h_bytes_per_step": nelem * 8 + B * C * 8,
                     "ms_per_step": e2e_ms, "api": "cawn_phase_accumulate_fwd_host (pinned host buffers)"},
             "gpu_launches": args.steps,
-            "clocks": clocks,
+            "clocks": clocks_now,
             "cpu_baseline": cpu,
         }
         print(json.dumps(line))
