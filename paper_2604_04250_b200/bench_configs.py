@@ -57,7 +57,7 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--only", default="", help="comma-separated subset of: mask,dynamic,cfg3,cfg4,cfg2")
+    ap.add_argument("--only", default="", help="comma-separated subset of: mask,dynamic,cfg3,cfg4,cfg2,decode")
     ap.add_argument("--cfg4-batch", type=int, default=0, help="batch rows of the config-4 run (0: the config's 16)")
     args = ap.parse_args()
     only = set(x for x in args.only.split(",") if x)
@@ -100,6 +100,33 @@ def main():
         _cfg4(args, cb, inputs, dev, IND)
     if want("cfg2"):
         _cfg2(args, cb, inputs, dev, IND)
+    if want("decode"):
+        _decode(args, cb, inputs, dev)
+
+
+def _decode(args, cb, inputs, dev):
+    import torch
+    # ---- single-token decode: L = 1 fused calls, state blob carried in place ------------------------
+    cfg = inputs.CONFIGS[4]
+    B, C, n = 1, cfg.C, 256
+    d = inputs.fused_inputs(B, n, C, cfg.seed, cfg.conv_k)
+    g, t, w = dev(d["gamma"]), dev(d["theta"]), dev(d["conv_w"])
+    prm = cb.make_params(B, 1, cfg.H, cfg.F, gate_eps=cfg.gate_eps, gate_tau=float(inputs.gate_tau(cfg.gate_eps)),
+                         conv_k=cfg.conv_k)
+    ws = cb.new_workspace(prm, cb.CAWN_OP_FWD)
+    nbytes = cb.cawn_workspace_bytes(prm, cb.CAWN_OP_STATE)
+    blob = torch.zeros(nbytes, dtype=torch.uint8, device="cuda")
+    h = dev(d["h"])
+    rows = [h[:, i:i + 1].contiguous() for i in range(n)]
+    y = torch.empty((B, 1, C), dtype=torch.complex64, device="cuda")
+
+    def gen(i):
+        for j in range(n):
+            cb.cawn_phase_accumulate_fwd(prm, rows[j], g, t, y, ws, conv_w=w, state_in=blob, state_out=blob)
+    ms = _time(gen, max(args.steps // 10, 3), 2)
+    assert cb.cawn_poll_status(ws) == 0
+    _report("decode_fused_B1_L1", n, n * C * 12, ms, n, {"us_per_token": ms * 1e3 / n,
+            "note": "one launch per token; latency-bound, bandwidth figures are not meaningful"})
 
 
 def _cfg3(args, cb, inputs, dev):
