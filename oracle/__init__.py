@@ -11,7 +11,8 @@ Functions mirror the steps of the path:
 * :func:`prelude`     causal depthwise conv -> phasor map -> gate -> push
 * :func:`scan`        the recurrence of Eq. (phase_accum_r/i), clamp, state
 * :func:`scan_bwd`    reverse-time adjoint with parameter gradients
-* :func:`forward`, :func:`fused_forward`  compositions of the above
+* :func:`prelude_bwd` backward of the prelude (conv, phasor map, straight-through gate)
+* :func:`forward`, :func:`fused_forward`, :func:`fused_backward`  compositions of the above
 
 No function here is "parity unpinned": see ``tests/test_oracle_*.py``.
 """
@@ -197,3 +198,36 @@ def fused_forward(h, w, gamma, theta, gate_eps, gate_tau, bias=None,
     z, mask, tail = prelude(h, w, bias, clamp_silu, tail_in, gate_eps, gate_tau)
     y, so = scan(z, theta, gamma=gamma, state_in=state_in, clamp_abs=clamp_abs)
     return y, so, mask, tail
+
+
+def prelude_bwd(h, w, dz, bias=None, clamp_silu=False, tail_in=None, gate_eps=0.0, gate_tau=-np.inf,
+                dtail_out=None):
+    """Backward of :func:`prelude` for a push gradient ``dz`` [B,L,C] complex.
+
+    Returns a dict with dh [B,L,C], dw [C,Kc], dbias [C], dtail_in [B,Kc-1,C] (float64)."""
+    hh, ww, bb, ti = _f32(h), _f32(w), _f32(bias), _f32(tail_in)
+    B, L, C = hh.shape
+    Kc = ww.shape[1]
+    dzz = _as_pairs(np.asarray(dz, dtype=np.complex128), np.float64)
+    dto = _f64(dtail_out)
+    dh = np.empty((B, L, C), np.float64)
+    dw = np.empty((C, Kc), np.float64)
+    db = np.empty(C, np.float64)
+    dti = np.empty((B, Kc - 1, C), np.float64)
+    _load().cawn_oracle_prelude_bwd(
+        ctypes.c_int(B), ctypes.c_int64(L), ctypes.c_int(C),
+        _ptr(hh, np.float32), _ptr(ww, np.float32), _ptr(bb, np.float32),
+        ctypes.c_int(Kc), ctypes.c_int(int(bool(clamp_silu))),
+        _ptr(ti, np.float32), ctypes.c_float(gate_eps), ctypes.c_float(gate_tau),
+        _ptr(dzz, np.float64), _ptr(dto, np.float64),
+        _ptr(dh, np.float64), _ptr(dw, np.float64), _ptr(db, np.float64), _ptr(dti, np.float64))
+    return {"dh": dh, "dw": dw, "dbias": db, "dtail_in": dti}
+
+
+def fused_backward(h, w, gamma, theta, G, gate_eps, gate_tau, bias=None, clamp_silu=False, tail_in=None,
+                   state_in=None, dstate_out=None, dtail_out=None):
+    """prelude -> scan forward, then scan_bwd -> prelude_bwd.  Returns the union of both dicts."""
+    z, mask, _ = prelude(h, w, bias, clamp_silu, tail_in, gate_eps, gate_tau)
+    out = scan_bwd(z, theta, G, gamma=gamma, state_in=state_in, dstate_out=dstate_out)
+    out.update(prelude_bwd(h, w, out["dp"], bias, clamp_silu, tail_in, gate_eps, gate_tau, dtail_out))
+    return out

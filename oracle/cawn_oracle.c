@@ -20,8 +20,10 @@
  * Pins (see tests/test_oracle_*.py): complex geometric series, prefix sum,
  * impulse response, brute-force O(L^2) weighted sums, scipy.signal.lfilter,
  * linearity, chunked == unchunked, gate ties, causal FIR, adjoint identity,
- * brute-force adjoint and central finite differences.  No function in this
- * file is "parity unpinned".
+ * brute-force adjoint and central finite differences (also of the fused path's
+ * backward, whose straight-through rule is pinned as a projection identity and
+ * whose chunked form is pinned against the unchunked one).  No function in
+ * this file is "parity unpinned".
  */
 #include <math.h>
 #include <stddef.h>
@@ -299,4 +301,105 @@ void cawn_oracle_scan_bwd(int B, int64_t L, int H, int F,
             dgamma[j] = dgamma[j] > c ? c : (dgamma[j] < -c ? -c : dgamma[j]);
     }
     free(P);
+}
+
+/* ------------------------------------------------------------------------ */
+/* Backward of the prelude (cawn_oracle_prelude) for a given push gradient
+ * dz = dLoss/dz (complex, as cawn_oracle_scan_bwd returns it in dp).
+ *
+ * Chain, per (b, t, c), with u, x, m, phase and the gate decision recomputed
+ * exactly as the forward does:
+ *   z = m_used (cos ph, sin ph),  m_used = m if open else 0
+ *   Straight-through gate (Section "Multi-Head Dynamic Parameter Projection",
+ *   Hard-Threshold Gating: beta = beta_hard - sg(beta) + beta): the forward
+ *   value of the magnitude is the gated one, its derivative with respect to
+ *   the ungated magnitude is 1 whether the gate is open or not.  Hence
+ *     dm  = Re(conj(dz) e^{i ph})        = dz_r cos ph + dz_i sin ph   (unmasked)
+ *     dph = Re(conj(dz) i z)             = m_used (-dz_r sin ph + dz_i cos ph)
+ *   m = sigmoid(x), ph = pi tanh(x):
+ *     dx = dm m (1 - m) + dph pi (1 - tanh(x)^2)
+ *   optional clamp to [-50,50] then SiLU (x = silu(clamp(u))): the clamp passes
+ *   the gradient inside the closed interval, silu'(v) = s (1 + v (1 - s)),
+ *   s = sigmoid(v); otherwise du = dx.
+ *   conv: u_t = bias + sum_k w[c,k] hrow(t-(Kc-1)+k), hrow(s) = h[s] for s >= 0,
+ *   the carried tail for s < 0:
+ *     dbias[c] += du,  dw[c,k] += du hrow(s),  dh[s] += w[c,k] du  (s >= 0),
+ *     dtail_in[Kh+s] += w[c,k] du (s < 0).
+ * dtail_out (optional, [B,Kc-1,C]) is the gradient arriving on this call's
+ * tail_out, i.e. on its last Kc-1 hidden rows as seen by the NEXT call: it is
+ * added to dh of those rows (and, when the call is shorter than Kc-1, to
+ * dtail_in of the rows it passed through).
+ * Outputs dh [B,L,C], dw [C,Kc], dbias [C] (may be NULL), dtail_in (may be
+ * NULL), all double, all overwritten.                                        */
+ORACLE_API
+void cawn_oracle_prelude_bwd(int B, int64_t L, int C,
+                             const float *h, const float *w, const float *bias,
+                             int Kc, int clamp_silu,
+                             const float *tail_in, float gate_eps, float gate_tau,
+                             const double *dz, const double *dtail_out,
+                             double *dh, double *dw, double *dbias, double *dtail_in)
+{
+    const double PI = 3.14159265358979323846;
+    const int Kh = Kc - 1;
+    memset(dh, 0, sizeof(double) * (size_t)B * (size_t)L * (size_t)C);
+    memset(dw, 0, sizeof(double) * (size_t)C * (size_t)Kc);
+    if (dbias) memset(dbias, 0, sizeof(double) * (size_t)C);
+    if (dtail_in) memset(dtail_in, 0, sizeof(double) * (size_t)B * (size_t)Kh * (size_t)C);
+    for (int b = 0; b < B; ++b) {
+        for (int64_t t = 0; t < L; ++t) {
+            for (int c = 0; c < C; ++c) {
+                double u = bias ? (double)bias[c] : 0.0;
+                float u32 = bias ? bias[c] : 0.0f;
+                for (int k = 0; k < Kc; ++k) {
+                    const int64_t s = t - Kh + k;
+                    float hv;
+                    if (s >= 0)       hv = h[((int64_t)b * L + s) * C + c];
+                    else if (tail_in) hv = tail_in[((int64_t)b * Kh + (Kh + s)) * C + c];
+                    else              hv = 0.0f;
+                    u  += (double)w[(int64_t)c * Kc + k] * (double)hv;
+                    u32 = fmaf(w[(int64_t)c * Kc + k], hv, u32);
+                }
+                double x = u, dxdu = 1.0;
+                if (clamp_silu) {
+                    const double v = u > 50.0 ? 50.0 : (u < -50.0 ? -50.0 : u);
+                    const double sg = 1.0 / (1.0 + exp(-v));
+                    x = v * sg;
+                    dxdu = (u >= -50.0 && u <= 50.0) ? sg * (1.0 + v * (1.0 - sg)) : 0.0;
+                }
+                const double m  = 1.0 / (1.0 + exp(-x));
+                const double th = tanh(x);
+                const double ph = PI * th;
+                const int open = clamp_silu ? (m >= (double)gate_eps) : (u32 >= gate_tau);
+                const int64_t e = ((int64_t)b * L + t) * C + c;
+                const double dzr = dz[2 * e], dzi = dz[2 * e + 1];
+                const double cs = cos(ph), sn = sin(ph);
+                const double dm  = dzr * cs + dzi * sn;
+                const double dph = (open ? m : 0.0) * (-dzr * sn + dzi * cs);
+                const double dx  = dm * m * (1.0 - m) + dph * PI * (1.0 - th * th);
+                const double du  = dx * dxdu;
+                if (dbias) dbias[c] += du;
+                for (int k = 0; k < Kc; ++k) {
+                    const int64_t s = t - Kh + k;
+                    const double wk = (double)w[(int64_t)c * Kc + k];
+                    if (s >= 0) {
+                        dw[(int64_t)c * Kc + k] += du * (double)h[((int64_t)b * L + s) * C + c];
+                        dh[((int64_t)b * L + s) * C + c] += wk * du;
+                    } else {
+                        if (tail_in)
+                            dw[(int64_t)c * Kc + k] += du * (double)tail_in[((int64_t)b * Kh + (Kh + s)) * C + c];
+                        if (dtail_in) dtail_in[((int64_t)b * Kh + (Kh + s)) * C + c] += wk * du;
+                    }
+                }
+            }
+        }
+        if (dtail_out)
+            for (int r = 0; r < Kh; ++r) {
+                const int64_t s = L - Kh + r;          /* the hidden row tail_out[r] holds */
+                for (int c = 0; c < C; ++c) {
+                    const double g = dtail_out[((int64_t)b * Kh + r) * C + c];
+                    if (s >= 0) dh[((int64_t)b * L + s) * C + c] += g;
+                    else if (dtail_in) dtail_in[((int64_t)b * Kh + (Kh + s)) * C + c] += g;
+                }
+            }
+    }
 }
