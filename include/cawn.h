@@ -79,7 +79,8 @@ enum {
     CAWN_OP_BWD_SAVED  = 1,  /* workspace of cawn_phase_accumulate_bwd with CAWN_SAVED_STATES    */
     CAWN_OP_BWD_PUSHES = 2,  /* ... with CAWN_SAVED_PUSHES (adds room for the recomputed states) */
     CAWN_OP_STATE      = 3,  /* size of one state blob                                           */
-    CAWN_OP_FWD_HOST   = 4   /* device staging + workspace of cawn_phase_accumulate_fwd_host     */
+    CAWN_OP_FWD_HOST   = 4,  /* device staging + workspace of cawn_phase_accumulate_fwd_host     */
+    CAWN_OP_MIXING_BWD = 5   /* workspace of cawn_mixing_bwd                                     */
 };
 
 /* What the backward was given to rebuild P_{t-1} from. */
@@ -199,6 +200,37 @@ CAWN_API int cawn_phase_accumulate_bwd_dynamic(const cawn_params *params,
                                                void *grad_state_in,
                                                void *workspace, size_t workspace_bytes,
                                                void *cuda_stream);
+
+/*
+ * Backward of the fused Resonance mixing path (cawn_phase_accumulate_fwd with conv_k >= 1,
+ * static retention): reverse scan, then the prelude's chain rule.
+ *   lam   = reverse scan of grad_y (as cawn_phase_accumulate_bwd); it is the gradient of the pushes
+ *   magnitude m = sigmoid(x), phase ph = pi tanh(x), push z = m_used (cos ph, sin ph):
+ *     d m  = Re(conj(lam) e^{i ph})                    straight-through: flows open or closed
+ *     d ph = m_used (-lam_r sin ph + lam_i cos ph)     m_used = m if the gate is open else 0
+ *   (the paper's hard-threshold gate with straight-through estimator, Section "Multi-Head Dynamic
+ *   Parameter Projection"), through the optional clamp + SiLU and the causal depthwise conv
+ *   (Section "Temporal Syntax Cache") to h, conv_w, conv_bias and the carried conv history.
+ * h [B,L,C] float, conv_w [C,conv_k], conv_bias [C] or NULL, gamma/theta [C]: as in the forward.
+ * saved_states: the forward's UNCLAMPED y [B,L,C] complex64; may be NULL when neither grad_gamma
+ *               nor grad_theta is wanted.
+ * state_in:     the forward's state blob (its conv history is read) or NULL.
+ * grad_y [B,L,C] complex64; grad_state_out: gradient of the forward's state_out blob (state part
+ *               and conv-history part, e.g. the next chunk's grad_state_in) or NULL.
+ * grad_h [B,L,C] float; grad_conv_w [C,conv_k], grad_conv_bias [C], grad_gamma [C], grad_theta [C]
+ *               float or NULL; grad_state_in: state blob of gradients or NULL.  All device.
+ * workspace:    >= cawn_workspace_bytes(CAWN_OP_MIXING_BWD), initialised once; it also holds the
+ *               push gradient lam (B*L*C complex64) between the two kernels.
+ * Deterministic (parameter sums: per-CTA partials combined in a fixed order in double).
+ */
+CAWN_API int cawn_mixing_bwd(const cawn_params *params,
+                             const float *h, const float *conv_w, const float *conv_bias,
+                             const float *gamma, const float *theta,
+                             const void *saved_states, const void *state_in,
+                             const void *grad_y, const void *grad_state_out,
+                             float *grad_h, float *grad_conv_w, float *grad_conv_bias,
+                             float *grad_gamma, float *grad_theta, void *grad_state_in,
+                             void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
  * Associative combine of two segment summaries (static retention):

@@ -28,14 +28,14 @@ CAWN_FLAG_PRELUDE_CLAMP_SILU = 1
 CAWN_FLAG_RETENTION_DYNAMIC = 2
 CAWN_FLAG_INPUT_INDEPENDENT = 4
 
-CAWN_OP_FWD, CAWN_OP_BWD_SAVED, CAWN_OP_BWD_PUSHES, CAWN_OP_STATE, CAWN_OP_FWD_HOST = range(5)
+CAWN_OP_FWD, CAWN_OP_BWD_SAVED, CAWN_OP_BWD_PUSHES, CAWN_OP_STATE, CAWN_OP_FWD_HOST, CAWN_OP_MIXING_BWD = range(6)
 CAWN_SAVED_STATES, CAWN_SAVED_PUSHES = 0, 1
 
 EXPORTS = (
     "cawn_status_string", "cawn_workspace_bytes", "cawn_workspace_init",
     "cawn_phase_accumulate_fwd", "cawn_phase_accumulate_bwd", "cawn_state_carry",
     "cawn_poll_status", "cawn_phase_accumulate_fwd_host", "cawn_phase_accumulate_fwd_static",
-    "cawn_phase_accumulate_bwd_dynamic",
+    "cawn_phase_accumulate_bwd_dynamic", "cawn_mixing_bwd",
 )
 
 
@@ -82,6 +82,7 @@ def lib():
         L.cawn_phase_accumulate_fwd.argtypes = [pp, vp, fp, fp, fp, fp, fp, fp, vp, vp, vp, vp, vp, sz, vp]
         L.cawn_phase_accumulate_bwd.argtypes = [pp, vp, ctypes.c_int, fp, fp, vp, vp, vp, vp, fp, fp, vp, vp, sz, vp]
         L.cawn_phase_accumulate_bwd_dynamic.argtypes = [pp, vp, ctypes.c_int, fp, fp, fp, vp, vp, vp, vp, fp, fp, fp, vp, vp, sz, vp]
+        L.cawn_mixing_bwd.argtypes = [pp, fp, fp, fp, fp, fp, vp, vp, vp, vp, fp, fp, fp, fp, fp, vp, vp, sz, vp]
         L.cawn_state_carry.argtypes = [pp, vp, vp, ctypes.c_int64, fp, fp, vp, vp]
         L.cawn_poll_status.argtypes = [vp, vp]
         L.cawn_phase_accumulate_fwd_host.argtypes = [pp, vp, fp, fp, vp, vp, vp, vp, vp, sz, vp]
@@ -202,3 +203,13 @@ def cawn_phase_accumulate_bwd_dynamic(params, saved, saved_kind, gamma_logit, fr
         _dp(state_in), _dp(grad_y), _dp(grad_state_out), _dp(grad_p), _dp(grad_gamma_logit),
         _dp(grad_freq_bias), _dp(grad_theta), _dp(grad_state_in), _dp(workspace),
         workspace.numel() * workspace.element_size(), _stream(stream)), "cawn_phase_accumulate_bwd_dynamic")
+
+
+def cawn_mixing_bwd(params, h, conv_w, gamma, theta, grad_y, grad_h, workspace, conv_bias=None, saved_states=None,
+                    state_in=None, grad_state_out=None, grad_conv_w=None, grad_conv_bias=None, grad_gamma=None,
+                    grad_theta=None, grad_state_in=None, stream=None):
+    _check(lib().cawn_mixing_bwd(
+        ctypes.byref(params), _dp(h), _dp(conv_w), _dp(conv_bias), _dp(gamma), _dp(theta), _dp(saved_states),
+        _dp(state_in), _dp(grad_y), _dp(grad_state_out), _dp(grad_h), _dp(grad_conv_w), _dp(grad_conv_bias),
+        _dp(grad_gamma), _dp(grad_theta), _dp(grad_state_in), _dp(workspace),
+        workspace.numel() * workspace.element_size(), _stream(stream)), "cawn_mixing_bwd")

@@ -1,6 +1,7 @@
 // libcawn: C-ABI entry points, argument validation, workspace layout and kernel launches.
 #include "../../include/cawn.h"
 #include "cawn_scan.cuh"
+#include "cawn_prelude_bwd.cuh"
 
 #include <math.h>
 #include <string.h>
@@ -270,6 +271,18 @@ int cawn_workspace_bytes(const cawn_params *params, int op, size_t *bytes)
         *bytes = total;
         return CAWN_OK;
     }
+    case CAWN_OP_MIXING_BWD: {
+        cawn_params q = *params;
+        q.conv_k = 0;                                   // the scan part is the Cartesian backward
+        size_t scan = 0;
+        const int rc2 = cawn_workspace_bytes(&q, CAWN_OP_BWD_SAVED, &scan);
+        if (rc2 != CAWN_OK) return rc2;
+        const int64_t rows_per_cta = (int64_t)kPbRows * kPbWarps;
+        const size_t rt = (size_t)((params->L + rows_per_cta - 1) / rows_per_cta);
+        *bytes = round_up(scan, 256) + round_up(n * sizeof(float2), 256) +
+                 round_up((size_t)params->B * (rt ? rt : 1) * (size_t)params->H * params->F * 5 * sizeof(float), 256);
+        return CAWN_OK;
+    }
     case CAWN_OP_STATE:
         *bytes = state_blob_bytes(params);
         return CAWN_OK;
@@ -508,6 +521,87 @@ int cawn_phase_accumulate_bwd_dynamic(const cawn_params *params, const void *sav
     return bwd_common(params, true, saved, saved_kind, nullptr, gamma_logit, freq_bias, theta, state_in, grad_y,
                       grad_state_out, grad_p, nullptr, grad_gamma_logit, grad_freq_bias, grad_theta,
                       grad_state_in, workspace, workspace_bytes, cuda_stream);
+}
+
+int cawn_mixing_bwd(const cawn_params *params, const float *h, const float *conv_w, const float *conv_bias,
+                    const float *gamma, const float *theta, const void *saved_states, const void *state_in,
+                    const void *grad_y, const void *grad_state_out, float *grad_h, float *grad_conv_w,
+                    float *grad_conv_bias, float *grad_gamma, float *grad_theta, void *grad_state_in,
+                    void *workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    int rc = check_params(params);
+    if (rc != CAWN_OK) return rc;
+    if (params->conv_k < 1 || params->conv_k > 4 || (params->flags & CAWN_FLAG_RETENTION_DYNAMIC))
+        return CAWN_ERR_UNSUPPORTED;
+    if ((params->flags & CAWN_FLAG_PRELUDE_CLAMP_SILU) && params->gate_eps > 0.4f) return CAWN_ERR_UNSUPPORTED;
+    if (conv_w == nullptr || gamma == nullptr || theta == nullptr || workspace == nullptr) return CAWN_ERR_NULL_POINTER;
+    if (params->L > 0 && (h == nullptr || grad_y == nullptr || grad_h == nullptr)) return CAWN_ERR_NULL_POINTER;
+    if (!aligned(h, 16) || !aligned(grad_h, 16) || !aligned(workspace, 16) || !aligned(state_in, 16) ||
+        !aligned(grad_state_out, 16) || !aligned(grad_state_in, 16))
+        return CAWN_ERR_MISALIGNED;
+    size_t need = 0;
+    rc = cawn_workspace_bytes(params, CAWN_OP_MIXING_BWD, &need);
+    if (rc != CAWN_OK) return rc;
+    if (workspace_bytes < need) return CAWN_ERR_WORKSPACE_TOO_SMALL;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    const int C = params->H * params->F, Kc = params->conv_k, Kh = Kc - 1;
+    const size_t n = (size_t)params->B * (size_t)params->L * C;
+    const size_t tail_off = round_up((size_t)params->B * C * sizeof(float2), 16);
+
+    // 1. reverse scan: lam into the workspace, grad_gamma / grad_theta / the state part of grad_state_in
+    cawn_params q = *params;
+    q.conv_k = 0;
+    size_t scan_bytes = 0;
+    rc = cawn_workspace_bytes(&q, CAWN_OP_BWD_SAVED, &scan_bytes);
+    if (rc != CAWN_OK) return rc;
+    char *base = reinterpret_cast<char *>(workspace);
+    float2 *lam = reinterpret_cast<float2 *>(base + round_up(scan_bytes, 256));
+    float *part = reinterpret_cast<float *>(base + round_up(scan_bytes, 256) + round_up(n * sizeof(float2), 256));
+    rc = bwd_common(&q, false, saved_states, CAWN_SAVED_STATES, gamma, nullptr, nullptr, theta, state_in, grad_y,
+                    grad_state_out, lam, grad_gamma, nullptr, nullptr, grad_theta, grad_state_in,
+                    workspace, scan_bytes, st);
+    if (rc != CAWN_OK) return rc;
+
+    // 2. the prelude's chain rule
+    const int64_t rows_per_cta = (int64_t)kPbRows * kPbWarps;
+    const int RT = (int)((params->L + rows_per_cta - 1) / rows_per_cta);
+    if (params->L > 0) {
+        if (RT > 65535 || params->B > 65535) return CAWN_ERR_UNSUPPORTED;
+        PreludeBwdParams pp;
+        memset(&pp, 0, sizeof(pp));
+        pp.h = h; pp.lam = lam; pp.conv_w = conv_w; pp.conv_bias = conv_bias;
+        if (Kh > 0) {
+            pp.tail_in = state_in ? reinterpret_cast<const float *>(reinterpret_cast<const char *>(state_in) + tail_off) : nullptr;
+            pp.dtail_out = grad_state_out ? reinterpret_cast<const float *>(reinterpret_cast<const char *>(grad_state_out) + tail_off) : nullptr;
+            pp.dtail_in = grad_state_in ? reinterpret_cast<float *>(reinterpret_cast<char *>(grad_state_in) + tail_off) : nullptr;
+        }
+        pp.dh = grad_h; pp.part = part;
+        pp.L = params->L; pp.B = params->B; pp.C = C; pp.G = (C + 63) / 64; pp.RT = RT; pp.Kc = Kc;
+        pp.clamp_silu = (params->flags & CAWN_FLAG_PRELUDE_CLAMP_SILU) ? 1 : 0;
+        pp.gate_tau = params->gate_tau;
+        const dim3 grid((unsigned)pp.G, (unsigned)params->B, (unsigned)RT);
+        if (C % 2 == 0) cawn_prelude_bwd_kernel<true><<<grid, kPbWarps * 32, 0, st>>>(pp);
+        else            cawn_prelude_bwd_kernel<false><<<grid, kPbWarps * 32, 0, st>>>(pp);
+        if (cudaGetLastError() != cudaSuccess) return CAWN_ERR_CUDA;
+        if (grad_conv_w != nullptr || grad_conv_bias != nullptr) {
+            const int warps = 8;
+            cawn_prelude_bwd_finalize_kernel<<<(C + warps - 1) / warps, warps * 32, 0, st>>>(
+                part, params->B * RT, C, Kc, grad_conv_w, grad_conv_bias);
+            if (cudaGetLastError() != cudaSuccess) return CAWN_ERR_CUDA;
+        }
+    } else {
+        // nothing ran: the incoming history gradient passes through, the parameter gradients are zero
+        if (grad_conv_w && cudaMemsetAsync(grad_conv_w, 0, (size_t)C * Kc * sizeof(float), st) != cudaSuccess) return CAWN_ERR_CUDA;
+        if (grad_conv_bias && cudaMemsetAsync(grad_conv_bias, 0, (size_t)C * sizeof(float), st) != cudaSuccess) return CAWN_ERR_CUDA;
+        if (grad_state_in != nullptr && Kh > 0) {
+            char *dst = reinterpret_cast<char *>(grad_state_in) + tail_off;
+            const size_t nb = (size_t)params->B * Kh * C * sizeof(float);
+            cudaError_t e = grad_state_out ? cudaMemcpyAsync(dst, reinterpret_cast<const char *>(grad_state_out) + tail_off, nb, cudaMemcpyDeviceToDevice, st)
+                                           : cudaMemsetAsync(dst, 0, nb, st);
+            if (e != cudaSuccess) return CAWN_ERR_CUDA;
+        }
+    }
+    return CAWN_OK;
 }
 
 int cawn_state_carry(const cawn_params *params, const void *state_prev, const void *state_local,
