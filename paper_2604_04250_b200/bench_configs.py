@@ -57,7 +57,7 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--only", default="", help="comma-separated subset of: mask,dynamic,cfg3,cfg4,cfg2,decode")
+    ap.add_argument("--only", default="", help="comma-separated subset of: mask,dynamic,cfg3,cfg4,cfg4bwd,cfg2,decode")
     ap.add_argument("--cfg4-batch", type=int, default=0, help="batch rows of the config-4 run (0: the config's 16)")
     args = ap.parse_args()
     only = set(x for x in args.only.split(",") if x)
@@ -98,6 +98,8 @@ def main():
         _cfg3(args, cb, inputs, dev)
     if want("cfg4"):
         _cfg4(args, cb, inputs, dev, IND)
+    if want("cfg4bwd"):
+        _cfg4_bwd(args, cb, inputs, dev)
     if want("cfg2"):
         _cfg2(args, cb, inputs, dev, IND)
     if want("decode"):
@@ -171,6 +173,33 @@ def _cfg4(args, cb, inputs, dev, IND):
                max(args.steps // 2, 5), args.warmup)
     assert cb.cawn_poll_status(ws) == 0
     _report("cfg4_fused" if B == cfg.B else "cfg4_fused_B%d" % B, B * L, B * L * C * 12, ms, 1)
+
+
+def _cfg4_bwd(args, cb, inputs, dev):
+    import torch
+    # ---- config 4, backward of the fused mixing path (saved states) -------------------------------
+    cfg = inputs.CONFIGS[4]
+    B, L, C = (args.cfg4_batch or cfg.B), cfg.L, cfg.C
+    d = inputs.fused_inputs(B, L, C, cfg.seed, cfg.conv_k, cfg.gamma_lo, cfg.gamma_hi)
+    g, t, w, h = dev(d["gamma"]), dev(d["theta"]), dev(d["conv_w"]), dev(d["h"])
+    prm = cb.make_params(B, L, cfg.H, cfg.F, gate_eps=cfg.gate_eps, gate_tau=float(inputs.gate_tau(cfg.gate_eps)),
+                         conv_k=cfg.conv_k)
+    P = torch.empty((B, L, C), dtype=torch.complex64, device="cuda")
+    wf = cb.new_workspace(prm, cb.CAWN_OP_FWD)
+    cb.cawn_phase_accumulate_fwd(prm, h, g, t, P, wf, conv_w=w)
+    gy = torch.randn((B, L, C, 2), device="cuda").view(torch.float32)
+    gy = torch.view_as_complex(gy)
+    gh = torch.empty((B, L, C), device="cuda")
+    gw, gb = torch.empty((C, cfg.conv_k), device="cuda"), torch.empty(C, device="cuda")
+    gg, gt = torch.empty(C, device="cuda"), torch.empty(C, device="cuda")
+    wb = cb.new_workspace(prm, cb.CAWN_OP_MIXING_BWD)
+    ms = _time(lambda i: cb.cawn_mixing_bwd(prm, h, w, g, t, gy, gh, wb, saved_states=P, grad_conv_w=gw,
+                                            grad_conv_bias=gb, grad_gamma=gg, grad_theta=gt),
+               max(args.steps // 2, 5), args.warmup)
+    assert cb.cawn_poll_status(wb) == 0
+    # reads grad_y (8) + P (8) + h (4), writes grad_h (4); lambda (8 written + 8 read) is internal traffic
+    _report("cfg4_mixing_bwd" if B == cfg.B else "cfg4_mixing_bwd_B%d" % B, B * L, B * L * C * 24, ms, 4,
+            {"note": "algorithmic bytes exclude the workspace pass of the adjoint states (16 B/elem more)"})
 
 
 def _cfg2(args, cb, inputs, dev, IND):
