@@ -12,6 +12,8 @@ Functions mirror the steps of the path:
 * :func:`scan`        the recurrence of Eq. (phase_accum_r/i), clamp, state
 * :func:`scan_bwd`    reverse-time adjoint with parameter gradients
 * :func:`prelude_bwd` backward of the prelude (conv, phasor map, straight-through gate)
+* :func:`wave_synthesis`, :func:`ear_conv`  planar Z of Eq. (wave_synth) and the depthwise
+  convolution across the harmonics that opens the SwiGLU Ear
 * :func:`forward`, :func:`fused_forward`, :func:`fused_backward`  compositions of the above
 
 No function here is "parity unpinned": see ``tests/test_oracle_*.py``.
@@ -183,6 +185,46 @@ def scan_bwd(z, theta, G, gamma=None, gamma_logit=None, freq_bias=None, H=None,
         out["dgamma_logit"] = dgl
         out["dfreq_bias"] = dfb
     return out
+
+
+def wave_synthesis(y, H, K):
+    """Eq. (wave_synth): Z_t = Concat(P^(r)_t, P^(i)_t).  ``y`` [B,L,H*K] complex ->
+    Z [B,L,2,H,K] float64: all real parts (head-major), then all imaginary parts."""
+    y = np.asarray(y, dtype=np.complex128)
+    B, L, C = y.shape
+    assert C == H * K
+    Z = np.empty((B, L, 2, H, K), dtype=np.float64)
+    Z[:, :, 0] = y.real.reshape(B, L, H, K)
+    Z[:, :, 1] = y.imag.reshape(B, L, H, K)
+    return Z
+
+
+def ear_conv(y, ear_w, ear_bias, H, K):
+    """Front of the Convolutional SwiGLU Ear (Section "Projection to Hidden State"): Z is viewed
+    as 2H feature channels (real heads, then imaginary heads) over K positions (the harmonics),
+    and each channel is convolved along K with its own taps.
+
+    ``ear_w`` [2H, Ke] with Ke odd, ``ear_bias`` [2H] or None.  The paper gives neither Ke nor
+    the padding; taken here: zero padding of (Ke-1)/2 on both sides (output length K) and the
+    cross-correlation convention of a Conv1d layer,
+        out[q, k] = bias[q] + sum_j w[q, j] Z[q, k + j - (Ke-1)/2].
+    Returns Z_conv [B,L,2,H,K] float64 (flattening its last three axes gives the 2HK-wide row).
+    """
+    Z = wave_synthesis(y, H, K)
+    w = np.asarray(ear_w, dtype=np.float64)
+    Q, Ke = w.shape
+    assert Q == 2 * H and Ke % 2 == 1
+    r = (Ke - 1) // 2
+    B, L = Z.shape[:2]
+    Zq = Z.reshape(B, L, Q, K)
+    pad = np.zeros((B, L, Q, K + 2 * r), dtype=np.float64)
+    pad[..., r:r + K] = Zq
+    out = np.zeros((B, L, Q, K), dtype=np.float64)
+    if ear_bias is not None:
+        out += np.asarray(ear_bias, dtype=np.float64)[None, None, :, None]
+    for j in range(Ke):
+        out += w[None, None, :, j, None] * pad[..., j:j + K]
+    return out.reshape(B, L, 2, H, K)
 
 
 def forward(p, gamma, theta, gate_eps, state_in=None, clamp_abs=0.0, **kw):
