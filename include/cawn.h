@@ -233,6 +233,34 @@ CAWN_API int cawn_mixing_bwd(const cawn_params *params,
                              void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
+ * Forward with the front of the Convolutional SwiGLU Ear as the scan's epilogue (Eq. (wave_synth)
+ * and Section "Projection to Hidden State: The Convolutional SwiGLU Ear", the depth-wise 1-D
+ * convolution across the K harmonics).  Everything up to the clamped state y_t is
+ * cawn_phase_accumulate_fwd (Cartesian or fused input, static retention only); instead of
+ * storing y the kernel writes
+ *   Z_t = Concat(Re y_t, Im y_t)  viewed as 2H channels (real heads, then imaginary heads) x K
+ *   z_conv[b,t,q,k] = ear_bias[q] + sum_j ear_w[q,j] Z_t[q, k + j - (ear_k-1)/2],  zero outside 0..K-1
+ * The paper states neither the tap count nor the padding: taken as ear_k taps (1 or 3; other
+ * values -> CAWN_ERR_UNSUPPORTED) with zero padding on both sides, cross-correlation order as in a
+ * Conv1d layer.  ear_k = 1 with ear_w = 1 and no bias gives the planar Z itself.
+ * ear_w:   [2H, ear_k] float (device).  ear_bias: [2H] float (device) or NULL.
+ * z_conv:  [B, L, 2, H, K] float (device, 16-byte aligned), K = params->F; as many bytes as y.
+ * state_out (if given) still receives the unclamped, unconvolved P_{L-1} (and the conv history).
+ * Limits: K must divide 64 unless H*K <= 64 (a CTA owns 64 adjacent channels and does not read
+ * its neighbours' harmonics); CAWN_FLAG_RETENTION_DYNAMIC -> CAWN_ERR_UNSUPPORTED.
+ * Other arguments, ownership, stream order and status reporting as cawn_phase_accumulate_fwd.
+ */
+CAWN_API int cawn_phase_accumulate_fwd_ear(const cawn_params *params,
+                                           const void *input,
+                                           const float *gamma, const float *theta,
+                                           const float *conv_w, const float *conv_bias,
+                                           const void *state_in,
+                                           const float *ear_w, const float *ear_bias, int ear_k,
+                                           float *z_conv, void *state_out, uint32_t *gate_mask,
+                                           void *workspace, size_t workspace_bytes,
+                                           void *cuda_stream);
+
+/*
  * Associative combine of two segment summaries (static retention):
  *   state_out = a^n_steps * state_prev + state_local,   a_j = gamma_j e^{i theta_j}
  * where state_local is the end state of an n_steps-long segment run from a ZERO state.  This is

@@ -57,7 +57,7 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--only", default="", help="comma-separated subset of: mask,dynamic,cfg3,cfg4,cfg4bwd,cfg2,decode")
+    ap.add_argument("--only", default="", help="comma-separated subset of: mask,ear,dynamic,cfg3,cfg4,cfg4bwd,cfg2,decode")
     ap.add_argument("--cfg4-batch", type=int, default=0, help="batch rows of the config-4 run (0: the config's 16)")
     args = ap.parse_args()
     only = set(x for x in args.only.split(",") if x)
@@ -84,6 +84,12 @@ def main():
         ms = _time(lambda i: cb.cawn_phase_accumulate_fwd(prm, ps[i % NS], g, t, ys[i % NS], ws, gate_mask=masks[i % NS]),
                    args.steps, args.warmup)
         _report("cfg1_train_fwd+mask", B * L, B * L * C * (16 + 0.125), ms, 1)
+    if want("ear"):
+        ew, eb = torch.randn((2 * cfg.H, 3), device="cuda"), torch.randn(2 * cfg.H, device="cuda")
+        zs = [y.view(torch.float32).view(B, L, 2, C) for y in ys]      # planar rows are as long as interleaved ones
+        ms = _time(lambda i: cb.cawn_phase_accumulate_fwd_ear(prm, ps[i % NS], g, t, ew, 3, zs[i % NS], ws, ear_bias=eb),
+                   args.steps, args.warmup)
+        _report("cfg1_train_fwd+ear_conv", B * L, B * L * C * 16, ms, 1)
     if want("dynamic"):
         dd = inputs.dynamic_retention_inputs(B, L, cfg.H, cfg.F, 7)
         gl, fb = dev(dd["gamma_logit"]), dev(dd["freq_bias"])

@@ -35,7 +35,7 @@ EXPORTS = (
     "cawn_status_string", "cawn_workspace_bytes", "cawn_workspace_init",
     "cawn_phase_accumulate_fwd", "cawn_phase_accumulate_bwd", "cawn_state_carry",
     "cawn_poll_status", "cawn_phase_accumulate_fwd_host", "cawn_phase_accumulate_fwd_static",
-    "cawn_phase_accumulate_bwd_dynamic", "cawn_mixing_bwd",
+    "cawn_phase_accumulate_bwd_dynamic", "cawn_mixing_bwd", "cawn_phase_accumulate_fwd_ear",
 )
 
 
@@ -83,6 +83,7 @@ def lib():
         L.cawn_phase_accumulate_bwd.argtypes = [pp, vp, ctypes.c_int, fp, fp, vp, vp, vp, vp, fp, fp, vp, vp, sz, vp]
         L.cawn_phase_accumulate_bwd_dynamic.argtypes = [pp, vp, ctypes.c_int, fp, fp, fp, vp, vp, vp, vp, fp, fp, fp, vp, vp, sz, vp]
         L.cawn_mixing_bwd.argtypes = [pp, fp, fp, fp, fp, fp, vp, vp, vp, vp, fp, fp, fp, fp, fp, vp, vp, sz, vp]
+        L.cawn_phase_accumulate_fwd_ear.argtypes = [pp, vp, fp, fp, fp, fp, vp, fp, fp, ctypes.c_int, fp, vp, vp, vp, sz, vp]
         L.cawn_state_carry.argtypes = [pp, vp, vp, ctypes.c_int64, fp, fp, vp, vp]
         L.cawn_poll_status.argtypes = [vp, vp]
         L.cawn_phase_accumulate_fwd_host.argtypes = [pp, vp, fp, fp, vp, vp, vp, vp, vp, sz, vp]
@@ -153,6 +154,16 @@ def cawn_phase_accumulate_fwd(params, input, gamma, theta, y, workspace, conv_w=
         _dp(gamma_logit), _dp(freq_bias), _dp(state_in), _dp(y), _dp(state_out), _dp(gate_mask),
         _dp(workspace), workspace.numel() * workspace.element_size(), _stream(stream)),
         "cawn_phase_accumulate_fwd")
+
+
+def cawn_phase_accumulate_fwd_ear(params, input, gamma, theta, ear_w, ear_k, z_conv, workspace, ear_bias=None,
+                                  conv_w=None, conv_bias=None, state_in=None, state_out=None, gate_mask=None,
+                                  stream=None):
+    _check(lib().cawn_phase_accumulate_fwd_ear(
+        ctypes.byref(params), _dp(input), _dp(gamma), _dp(theta), _dp(conv_w), _dp(conv_bias), _dp(state_in),
+        _dp(ear_w), _dp(ear_bias), int(ear_k), _dp(z_conv), _dp(state_out), _dp(gate_mask),
+        _dp(workspace), workspace.numel() * workspace.element_size(), _stream(stream)),
+        "cawn_phase_accumulate_fwd_ear")
 
 
 def cawn_phase_accumulate_bwd(params, saved, saved_kind, gamma, theta, grad_y, grad_p, workspace,

@@ -100,7 +100,7 @@ inline bool grid_ok(const cawn_params *p, const Geometry &g)
 // The float4 path needs every row segment on a 16-byte boundary: C even (the arrays
 // themselves are checked to be 16-byte aligned).  The tile is staged in dynamic shared memory;
 // MINB is the number of CTAs per SM the register allocation leaves room for.
-template <int T, int W, int KIND, bool VEC, int MINB, bool DYN>
+template <int T, int W, int KIND, bool VEC, int MINB, bool DYN, bool EAR = false>
 cudaError_t launch_scan_inst(const ScanParams &sp, cudaStream_t st)
 {
     constexpr size_t smem = sizeof(ScanSmem<T, W, KIND, DYN>);
@@ -109,7 +109,7 @@ cudaError_t launch_scan_inst(const ScanParams &sp, cudaStream_t st)
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= 64 || !configured[dev]) {
-        e = cudaFuncSetAttribute(cawn_scan_kernel<T, W, KIND, VEC, MINB, DYN>,
+        e = cudaFuncSetAttribute(cawn_scan_kernel<T, W, KIND, VEC, MINB, DYN, EAR>,
                                  cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) configured[dev] = true;
@@ -127,13 +127,13 @@ cudaError_t launch_scan_inst(const ScanParams &sp, cudaStream_t st)
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, cawn_scan_kernel<T, W, KIND, VEC, MINB, DYN>, sp);
+    return cudaLaunchKernelEx(&cfg, cawn_scan_kernel<T, W, KIND, VEC, MINB, DYN, EAR>, sp);
 }
-template <int T, int W, int KIND, int MINB, bool DYN = false>
+template <int T, int W, int KIND, int MINB, bool DYN = false, bool EAR = false>
 cudaError_t launch_scan(const ScanParams &sp, cudaStream_t st)
 {
-    return sp.C % 2 == 0 ? launch_scan_inst<T, W, KIND, true, MINB, DYN>(sp, st)
-                         : launch_scan_inst<T, W, KIND, false, MINB, DYN>(sp, st);
+    return sp.C % 2 == 0 ? launch_scan_inst<T, W, KIND, true, MINB, DYN, EAR>(sp, st)
+                         : launch_scan_inst<T, W, KIND, false, MINB, DYN, EAR>(sp, st);
 }
 
 // First-wave stagger of the static forward scan: about two thirds of the time one SM's share of
@@ -164,6 +164,10 @@ void set_stagger(ScanParams &sp, TileShape ts)
 
 inline cudaError_t launch_fwd(TileShape ts, const ScanParams &sp, cudaStream_t st, bool dyn = false)
 {
+    if (sp.ear_w != nullptr) {
+        if (ts.T == 16) return launch_scan<16, 8, KIND_FWD, 3, false, true>(sp, st);
+        return launch_scan<4, 4, KIND_FWD, 8, false, true>(sp, st);
+    }
     if (dyn) {
         if (ts.T == 16) return launch_scan<16, 8, KIND_FWD, 2, true>(sp, st);
         return launch_scan<4, 4, KIND_FWD, 8, true>(sp, st);
@@ -173,6 +177,10 @@ inline cudaError_t launch_fwd(TileShape ts, const ScanParams &sp, cudaStream_t s
 }
 inline cudaError_t launch_fused(TileShape ts, const ScanParams &sp, cudaStream_t st)
 {
+    if (sp.ear_w != nullptr) {
+        if (ts.T == 16) return launch_scan<16, 8, KIND_FUSED, 3, false, true>(sp, st);
+        return launch_scan<4, 4, KIND_FUSED, 8, false, true>(sp, st);
+    }
     if (ts.T == 16) return launch_scan<16, 8, KIND_FUSED, 3>(sp, st);
     return launch_scan<4, 4, KIND_FUSED, 8>(sp, st);
 }
@@ -304,18 +312,26 @@ int cawn_workspace_init(void *workspace, size_t workspace_bytes, void *cuda_stre
     return CAWN_OK;
 }
 
-int cawn_phase_accumulate_fwd(const cawn_params *params, const void *input,
-                              const float *gamma, const float *theta,
-                              const float *conv_w, const float *conv_bias,
-                              const float *gamma_logit, const float *freq_bias,
-                              const void *state_in, void *y, void *state_out,
-                              uint32_t *gate_mask, void *workspace, size_t workspace_bytes,
-                              void *cuda_stream)
+// Forward, with (ear_w != NULL) or without the Ear epilogue.
+static int fwd_common(const cawn_params *params, const void *input,
+                      const float *gamma, const float *theta,
+                      const float *conv_w, const float *conv_bias,
+                      const float *gamma_logit, const float *freq_bias,
+                      const void *state_in, void *y, void *state_out,
+                      uint32_t *gate_mask, void *workspace, size_t workspace_bytes,
+                      void *cuda_stream, const float *ear_w, const float *ear_bias, int ear_k)
 {
     int rc = check_params(params);
     if (rc != CAWN_OK) return rc;
     const bool dyn = (params->flags & CAWN_FLAG_RETENTION_DYNAMIC) != 0;
     const bool fused = params->conv_k != 0;
+    if (ear_w != nullptr) {
+        if (ear_k != 1 && ear_k != 3) return CAWN_ERR_UNSUPPORTED;
+        if (dyn) return CAWN_ERR_UNSUPPORTED;
+        // a CTA owns 64 adjacent channels: a head's harmonics must not straddle two of them
+        if ((long long)params->H * params->F > 64 && 64 % params->F != 0) return CAWN_ERR_UNSUPPORTED;
+        if (!aligned(ear_w, 4) || !aligned(ear_bias, 4)) return CAWN_ERR_MISALIGNED;
+    }
     if (dyn) {
         if (fused) return CAWN_ERR_UNSUPPORTED;
         if (gamma_logit == nullptr || freq_bias == nullptr) return CAWN_ERR_NULL_POINTER;
@@ -364,6 +380,8 @@ int cawn_phase_accumulate_fwd(const cawn_params *params, const void *input,
     set_gate(sp, params->gate_eps);
     sp.clampv = params->clamp_abs > 0.f ? params->clamp_abs : 0.f;
     sp.poll_limit = kPollLimit;
+    sp.ear_w = ear_w; sp.ear_bias = ear_bias; sp.ear_k = ear_k;
+    sp.H = params->H; sp.F = params->F;
     if (fused) {
         // state blob: P [B,C] complex64, then (16-byte aligned) the conv history [B,conv_k-1,C]
         const size_t tail_off = round_up((size_t)params->B * g.C * sizeof(float2), 16);
@@ -384,6 +402,31 @@ int cawn_phase_accumulate_fwd(const cawn_params *params, const void *input,
     if (!dyn && ts.T == 16) set_stagger(sp, ts);
     if (launch_fwd(ts, sp, st, dyn) != cudaSuccess) return CAWN_ERR_CUDA;
     return CAWN_OK;
+}
+
+int cawn_phase_accumulate_fwd(const cawn_params *params, const void *input,
+                              const float *gamma, const float *theta,
+                              const float *conv_w, const float *conv_bias,
+                              const float *gamma_logit, const float *freq_bias,
+                              const void *state_in, void *y, void *state_out,
+                              uint32_t *gate_mask, void *workspace, size_t workspace_bytes,
+                              void *cuda_stream)
+{
+    return fwd_common(params, input, gamma, theta, conv_w, conv_bias, gamma_logit, freq_bias, state_in, y,
+                      state_out, gate_mask, workspace, workspace_bytes, cuda_stream, nullptr, nullptr, 0);
+}
+
+int cawn_phase_accumulate_fwd_ear(const cawn_params *params, const void *input,
+                                  const float *gamma, const float *theta,
+                                  const float *conv_w, const float *conv_bias,
+                                  const void *state_in,
+                                  const float *ear_w, const float *ear_bias, int ear_k,
+                                  float *z_conv, void *state_out, uint32_t *gate_mask,
+                                  void *workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    if (ear_w == nullptr) return CAWN_ERR_NULL_POINTER;
+    return fwd_common(params, input, gamma, theta, conv_w, conv_bias, nullptr, nullptr, state_in, z_conv,
+                      state_out, gate_mask, workspace, workspace_bytes, cuda_stream, ear_w, ear_bias, ear_k);
 }
 
 // Backward of the Cartesian forward, static (gamma) or time-varying (gamma_logit, freq_bias)

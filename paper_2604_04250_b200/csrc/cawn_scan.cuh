@@ -90,6 +90,12 @@ struct ScanParams {
     // so that the CTAs sharing an SM run out of phase and their load, arithmetic and store
     // phases overlap instead of alternating.  0 = off.
     int stagger_cycles, stagger_group, stagger_slots;
+    // Ear epilogue (EAR): instead of interleaved complex y, the kernel writes the planar row
+    // Z = (all real parts, all imaginary parts) [B,L,2,H,F] after a depthwise convolution along
+    // the F harmonics of each head (ear_k taps, zero padding, one tap set per (part, head)).
+    const float *ear_w;          // [2H][ear_k]
+    const float *ear_bias;       // [2H] or NULL
+    int ear_k;                   // 1 or 3
     int early_loads;             // the input rows may be fetched before the preceding launch on the
                                  // stream has finished (the caller vouches they are not its output)
 };
@@ -185,11 +191,12 @@ __device__ __forceinline__ void fetch_rows(float4 *dst, uint32_t dst_s, const ch
     }
 }
 
-template <int T, int W, int KIND, bool VEC, bool DYN, bool FULL>
+template <int T, int W, int KIND, bool VEC, bool DYN, bool FULL, bool EAR = false>
 __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, KIND, DYN> &sm,
                                           const int g, const int b, const int k)
 {
     static_assert(!(DYN && KIND == KIND_FUSED), "time-varying retention is not built for the fused path");
+    static_assert(!(EAR && (DYN || KIND == KIND_BWD)), "the Ear epilogue belongs to the static forward");
     constexpr bool REV = (KIND == KIND_BWD);
     constexpr int TILE = T * W;
     constexpr int M = kWindow;
@@ -649,8 +656,59 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
             else P = cfma2(aT, P, sm.sE[i][lane]);
         }
 
-        char *const rbase = reinterpret_cast<char *>(prm.out) + e0 * 8;
+        // EAR: a planar row is 2C floats, as long as an interleaved one; the real parts of this
+        // lane's two channels sit c0 floats into it, the imaginary parts C floats further
+        char *const rbase = reinterpret_cast<char *>(prm.out) + (EAR ? (e0 - c0) * 8 + c0 * 4 : e0 * 8);
         const float cl = prm.clampv;
+        // Ear taps of this lane's two channels, real and imaginary part: (left, centre, right,
+        // bias).  A tap whose source harmonic lies outside the head is zero (zero padding), so the
+        // values the shuffles bring in from a neighbouring head never count.
+        float ewr[2][4] = {}, ewi[2][4] = {};
+        if constexpr (EAR) {
+            const int Fh = prm.F, Ke = prm.ear_k, lead = (3 - Ke) / 2;
+#pragma unroll
+            for (int ch = 0; ch < 2; ++ch) {
+                const int c = c0 + ch;
+                if (c < C) {
+                    const int hh = c / Fh, kk = c - hh * Fh;
+#pragma unroll
+                    for (int j = 0; j < 3; ++j) {
+                        const int jj = j - lead, src = kk + j - 1;
+                        if (jj >= 0 && jj < Ke && src >= 0 && src < Fh) {
+                            ewr[ch][j] = prm.ear_w[hh * Ke + jj];
+                            ewi[ch][j] = prm.ear_w[(prm.H + hh) * Ke + jj];
+                        }
+                    }
+                    if (prm.ear_bias != nullptr) { ewr[ch][3] = prm.ear_bias[hh]; ewi[ch][3] = prm.ear_bias[prm.H + hh]; }
+                }
+            }
+        }
+        // one output row of this lane's channel pair; every lane of the warp takes part (the Ear
+        // form exchanges edge channels with the neighbouring lanes)
+        auto store_row = [&](int i, float4 o) {
+            char *r = const_cast<char *>(row_ptr(rbase, rowbytes, i));
+            if constexpr (EAR) {
+                const float lre = __shfl_up_sync(0xffffffffu, o.z, 1), lim = __shfl_up_sync(0xffffffffu, o.w, 1);
+                const float rre = __shfl_down_sync(0xffffffffu, o.x, 1), rim = __shfl_down_sync(0xffffffffu, o.y, 1);
+                const float zrA = fmaf(ewr[0][0], lre, fmaf(ewr[0][1], o.x, fmaf(ewr[0][2], o.z, ewr[0][3])));
+                const float zrB = fmaf(ewr[1][0], o.x, fmaf(ewr[1][1], o.z, fmaf(ewr[1][2], rre, ewr[1][3])));
+                const float ziA = fmaf(ewi[0][0], lim, fmaf(ewi[0][1], o.y, fmaf(ewi[0][2], o.w, ewi[0][3])));
+                const float ziB = fmaf(ewi[1][0], o.y, fmaf(ewi[1][1], o.w, fmaf(ewi[1][2], rim, ewi[1][3])));
+                float *zr = reinterpret_cast<float *>(r), *zi = zr + C;
+                if (VEC) {
+                    if (vA) { __stcs(reinterpret_cast<float2 *>(zr), make_float2(zrA, zrB)); __stcs(reinterpret_cast<float2 *>(zi), make_float2(ziA, ziB)); }
+                } else {
+                    if (vA) { __stcs(zr, zrA); __stcs(zi, ziA); }
+                    if (vB) { __stcs(zr + 1, zrB); __stcs(zi + 1, ziB); }
+                }
+            } else if (VEC) {
+                if (vA) __stcs(reinterpret_cast<float4 *>(r), o);
+            } else {
+                float2 *r2 = reinterpret_cast<float2 *>(r);
+                if (vA) __stcs(r2, make_float2(o.x, o.y));
+                if (vB) __stcs(r2 + 1, make_float2(o.z, o.w));
+            }
+        };
         // DYN: factor of the step into row i (forward: the row's own; backward: the factor of
         // the row processed before it), and the running sum of the logit gradient
         float2 gstep = make_float2(0.f, 0.f), sacc = make_float2(0.f, 0.f);
@@ -665,15 +723,7 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
                 } else {
                     P = cfma2(a, P, xs[i * 32]);
                 }
-                const float4 o = clamped ? clamp4(P, cl) : P;
-                char *r = const_cast<char *>(row_ptr(rbase, rowbytes, i));
-                if (VEC) {
-                    if (vA) __stcs(reinterpret_cast<float4 *>(r), o);
-                } else {
-                    float2 *r2 = reinterpret_cast<float2 *>(r);
-                    if (vA) __stcs(r2, make_float2(o.x, o.y));
-                    if (vB) __stcs(r2 + 1, make_float2(o.z, o.w));
-                }
+                store_row(i, clamped ? clamp4(P, cl) : P);
                 if constexpr (KIND == KIND_BWD) {
                     // conj(lam) * P_{t-1}
                     const float4 q = sm.tile[1][w * T + i][lane];
@@ -725,14 +775,7 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
                     Pr = nr; Pi = ni;
                     float4 o = make_float4(Pr.x, Pi.x, Pr.y, Pi.y);
                     if (cl > 0.f) o = clamp4(o, cl);
-                    char *r = const_cast<char *>(row_ptr(rbase, rowbytes, i));
-                    if (VEC) {
-                        if (vA) __stcs(reinterpret_cast<float4 *>(r), o);
-                    } else {
-                        float2 *r2 = reinterpret_cast<float2 *>(r);
-                        if (vA) __stcs(r2, make_float2(o.x, o.y));
-                        if (vB) __stcs(r2 + 1, make_float2(o.z, o.w));
-                    }
+                    store_row(i, o);
                 }
             }
             P = make_float4(Pr.x, Pi.x, Pr.y, Pi.y);
@@ -816,7 +859,7 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
     }
 }
 
-template <int T, int W, int KIND, bool VEC, int MINB, bool DYN = false>
+template <int T, int W, int KIND, bool VEC, int MINB, bool DYN = false, bool EAR = false>
 __global__ void __launch_bounds__(W * 32, MINB) cawn_scan_kernel(const ScanParams prm)
 {
     constexpr int TILE = T * W;
@@ -829,8 +872,8 @@ __global__ void __launch_bounds__(W * 32, MINB) cawn_scan_kernel(const ScanParam
     const int k = blockIdx.z;                         // tile index along (logical) time
     grid_launch_dependents();
     const bool full = ((long long)(k + 1) * TILE <= prm.L) && (g * 64 + 64 <= prm.C);
-    if (full) scan_tile<T, W, KIND, VEC, DYN, true>(prm, sm, g, b, k);
-    else      scan_tile<T, W, KIND, VEC, DYN, false>(prm, sm, g, b, k);
+    if (full) scan_tile<T, W, KIND, VEC, DYN, true, EAR>(prm, sm, g, b, k);
+    else      scan_tile<T, W, KIND, VEC, DYN, false, EAR>(prm, sm, g, b, k);
 }
 
 // grad_gamma_j = Re(e^{i theta} Q_j), grad_theta_j = -Im(a_j Q_j), Q_j = sum of the per-tile
