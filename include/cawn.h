@@ -62,7 +62,7 @@ typedef enum cawn_status {
 enum {
     CAWN_FLAG_PRELUDE_CLAMP_SILU = 1u << 0, /* fused path: clamp conv output to +-50, then SiLU   */
     CAWN_FLAG_RETENTION_DYNAMIC  = 1u << 1, /* gamma_t = sigmoid(gamma_logit[b,t,h] + freq_bias[k]) */
-    CAWN_FLAG_INPUT_INDEPENDENT  = 1u << 2  /* forward: the caller vouches that `input`, gamma, theta
+    CAWN_FLAG_INPUT_INDEPENDENT  = 1u << 2, /* forward: the caller vouches that `input`, gamma, theta
                                                (and the conv weights) are not written by the call
                                                made just before this one on the same stream.  The
                                                kernels are launched so that a call may start while the
@@ -71,6 +71,18 @@ enum {
                                                during that overlap.  States, masks, workspaces and all
                                                outputs are only touched once the previous call is
                                                complete, with or without the flag.                    */
+    CAWN_FLAG_INPUT_BF16         = 1u << 3, /* forward: `input` is stored as bfloat16 (Cartesian: pairs
+                                               (re, im) of bf16, 4 bytes per channel; fused path: one
+                                               bf16 per channel) and widened, exactly, to float on load */
+    CAWN_FLAG_OUTPUT_BF16        = 1u << 4  /* forward: `y` is stored as pairs (re, im) of bfloat16,
+                                               each component rounded to nearest even from the fp32
+                                               result.  With either flag the recurrence, the carried
+                                               state, state_out and the conv history stay fp32 (the
+                                               paper runs a bf16 network around an fp32 scan:
+                                               Section "Mixed-Precision and Float32
+                                               Stabilization").  Not available with the time-varying retention,
+                                               the Ear epilogue, the host-staged forward or any
+                                               backward: CAWN_ERR_UNSUPPORTED.                          */
 };
 
 /* Operation selector of cawn_workspace_bytes(). */

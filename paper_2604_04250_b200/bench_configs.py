@@ -57,7 +57,7 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--only", default="", help="comma-separated subset of: mask,ear,dynamic,cfg3,cfg4,cfg4bwd,cfg2,decode")
+    ap.add_argument("--only", default="", help="comma-separated subset of: mask,ear,bf16,dynamic,cfg3,cfg4,cfg4bwd,cfg2,decode")
     ap.add_argument("--cfg4-batch", type=int, default=0, help="batch rows of the config-4 run (0: the config's 16)")
     args = ap.parse_args()
     only = set(x for x in args.only.split(",") if x)
@@ -90,6 +90,16 @@ def main():
         ms = _time(lambda i: cb.cawn_phase_accumulate_fwd_ear(prm, ps[i % NS], g, t, ew, 3, zs[i % NS], ws, ear_bias=eb),
                    args.steps, args.warmup)
         _report("cfg1_train_fwd+ear_conv", B * L, B * L * C * 16, ms, 1)
+    if want("bf16"):
+        p16 = [p.view(torch.float32).to(torch.bfloat16).view(B, L, C, 2) for p in ps]
+        y16 = [torch.empty((B, L, C, 2), dtype=torch.bfloat16, device="cuda") for _ in range(NS)]
+        for name, fl, xin, yout, nbytes in (
+                ("cfg1_train_fwd_bf16_in+out", cb.CAWN_FLAG_INPUT_BF16 | cb.CAWN_FLAG_OUTPUT_BF16, p16, y16, 8),
+                ("cfg1_train_fwd_bf16_out", cb.CAWN_FLAG_OUTPUT_BF16, ps, y16, 12)):
+            prm16 = cb.make_params(B, L, cfg.H, cfg.F, gate_eps=cfg.gate_eps, flags=IND | fl)
+            ms = _time(lambda i: cb.cawn_phase_accumulate_fwd(prm16, xin[i % NS], g, t, yout[i % NS], ws), args.steps, args.warmup)
+            _report(name, B * L, B * L * C * nbytes, ms, 1)
+        del p16, y16
     if want("dynamic"):
         dd = inputs.dynamic_retention_inputs(B, L, cfg.H, cfg.F, 7)
         gl, fb = dev(dd["gamma_logit"]), dev(dd["freq_bias"])
@@ -179,6 +189,15 @@ def _cfg4(args, cb, inputs, dev, IND):
                max(args.steps // 2, 5), args.warmup)
     assert cb.cawn_poll_status(ws) == 0
     _report("cfg4_fused" if B == cfg.B else "cfg4_fused_B%d" % B, B * L, B * L * C * 12, ms, 1)
+    if "bf16" in args.only or not args.only:
+        prm16 = cb.make_params(B, L, cfg.H, cfg.F, gate_eps=cfg.gate_eps, gate_tau=float(inputs.gate_tau(cfg.gate_eps)),
+                               conv_k=cfg.conv_k, flags=IND | cb.CAWN_FLAG_INPUT_BF16 | cb.CAWN_FLAG_OUTPUT_BF16)
+        h16 = [h.to(torch.bfloat16) for h in hs]
+        y16 = [torch.empty((B, L, C, 2), dtype=torch.bfloat16, device="cuda") for _ in range(NS)]
+        ms = _time(lambda i: cb.cawn_phase_accumulate_fwd(prm16, h16[i % NS], g, t, y16[i % NS], ws, conv_w=w),
+                   max(args.steps // 2, 5), args.warmup)
+        assert cb.cawn_poll_status(ws) == 0
+        _report("cfg4_fused_bf16_in+out", B * L, B * L * C * 6, ms, 1)
 
 
 def _cfg4_bwd(args, cb, inputs, dev):

@@ -27,6 +27,8 @@ CAWN_ERR_CARRY_TIMEOUT = 1
 CAWN_FLAG_PRELUDE_CLAMP_SILU = 1
 CAWN_FLAG_RETENTION_DYNAMIC = 2
 CAWN_FLAG_INPUT_INDEPENDENT = 4
+CAWN_FLAG_INPUT_BF16 = 8
+CAWN_FLAG_OUTPUT_BF16 = 16
 
 CAWN_OP_FWD, CAWN_OP_BWD_SAVED, CAWN_OP_BWD_PUSHES, CAWN_OP_STATE, CAWN_OP_FWD_HOST, CAWN_OP_MIXING_BWD = range(6)
 CAWN_SAVED_STATES, CAWN_SAVED_PUSHES = 0, 1

@@ -13,8 +13,10 @@ INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-    "-Xcompiler", "-fPIC,-fvisibility=hidden", "-shared", "--cudart", "static",
+    "-Xcompiler", "-fPIC,-fvisibility=hidden",
 ]
+LINK_FLAGS = ["-shared", "--cudart", "static"]
+OBJ_DIR = os.path.join(HERE, "_build")
 
 
 def sources():
@@ -34,10 +36,31 @@ def build(force: bool = False, verbose: bool = False) -> str:
     if not force and not _stale():
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    tmp = LIB + ".tmp.%d" % os.getpid()
-    cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-o", tmp] + sources()
-    subprocess.check_call(cmd)
-    os.replace(tmp, LIB)
+    os.makedirs(OBJ_DIR, exist_ok=True)
+    tag = ".%d" % os.getpid()
+    jobs = []
+    for src in sources():                   # one nvcc per translation unit, side by side
+        obj = os.path.join(OBJ_DIR, os.path.basename(src)[:-3] + tag + ".o")
+        cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-c", "-o", obj, src]
+        jobs.append((src, obj, subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))
+    failed = []
+    for src, obj, proc in jobs:
+        out, _ = proc.communicate()
+        if out and (verbose or proc.returncode != 0):
+            sys.stderr.write(out)
+        if proc.returncode != 0:
+            failed.append(src)
+    objs = [obj for _, obj, _ in jobs]
+    try:
+        if failed:
+            raise RuntimeError("nvcc failed on: " + ", ".join(failed))
+        tmp = LIB + ".tmp" + tag
+        subprocess.check_call([nvcc] + NVCC_FLAGS + LINK_FLAGS + ["-o", tmp] + objs)
+        os.replace(tmp, LIB)
+    finally:
+        for obj in objs:
+            if os.path.exists(obj):
+                os.remove(obj)
     return LIB
 
 

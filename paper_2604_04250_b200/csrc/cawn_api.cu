@@ -1,6 +1,7 @@
 // libcawn: C-ABI entry points, argument validation, workspace layout and kernel launches.
 #include "../../include/cawn.h"
-#include "cawn_scan.cuh"
+#include "cawn_launch.cuh"
+#include "cawn_small_kernels.cuh"
 #include "cawn_prelude_bwd.cuh"
 
 #include <math.h>
@@ -15,9 +16,8 @@ constexpr unsigned kPollLimit = 1u << 20;   // ~1 s of polling before a carry wa
 inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 inline bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
-// Tile shape of the scan kernels.  Long calls use 128-step tiles (8 warps x 16 steps); short
-// ones (decode, tiny chunks) use 16-step tiles so that a call is not one mostly empty CTA.
-struct TileShape { int T, W; };
+// Long calls use 128-step tiles (8 warps x 16 steps); short ones (decode, tiny chunks) use
+// 16-step tiles so that a call is not one mostly empty CTA.
 inline TileShape fwd_shape(int64_t L) { return L > 32 ? TileShape{16, 8} : TileShape{4, 4}; }
 inline TileShape bwd_shape(int64_t L) { return L > 32 ? TileShape{8, 8} : TileShape{4, 4}; }
 
@@ -77,7 +77,8 @@ int check_params(const cawn_params *p)
     if (p->B < 1 || p->L < 0 || p->H < 1 || p->F < 1) return CAWN_ERR_INVALID_ARG;
     if ((int64_t)p->H * p->F > (1 << 24)) return CAWN_ERR_INVALID_ARG;
     if (p->conv_k < 0) return CAWN_ERR_INVALID_ARG;
-    if (p->flags & ~(uint32_t)(CAWN_FLAG_PRELUDE_CLAMP_SILU | CAWN_FLAG_RETENTION_DYNAMIC | CAWN_FLAG_INPUT_INDEPENDENT))
+    if (p->flags & ~(uint32_t)(CAWN_FLAG_PRELUDE_CLAMP_SILU | CAWN_FLAG_RETENTION_DYNAMIC | CAWN_FLAG_INPUT_INDEPENDENT |
+                                 CAWN_FLAG_INPUT_BF16 | CAWN_FLAG_OUTPUT_BF16))
         return CAWN_ERR_INVALID_ARG;
     if (!(p->gate_eps >= 0.f)) return CAWN_ERR_INVALID_ARG;
     return CAWN_OK;
@@ -95,45 +96,6 @@ size_t state_blob_bytes(const cawn_params *p)
 inline bool grid_ok(const cawn_params *p, const Geometry &g)
 {
     return p->B <= 65535 && g.K <= 65535 && (double)p->B * g.G * g.K < 4294967295.0;
-}
-
-// The float4 path needs every row segment on a 16-byte boundary: C even (the arrays
-// themselves are checked to be 16-byte aligned).  The tile is staged in dynamic shared memory;
-// MINB is the number of CTAs per SM the register allocation leaves room for.
-template <int T, int W, int KIND, bool VEC, int MINB, bool DYN, bool EAR = false>
-cudaError_t launch_scan_inst(const ScanParams &sp, cudaStream_t st)
-{
-    constexpr size_t smem = sizeof(ScanSmem<T, W, KIND, DYN>);
-    static bool configured[64] = {};
-    int dev = 0;
-    cudaError_t e = cudaGetDevice(&dev);
-    if (e != cudaSuccess) return e;
-    if (dev < 0 || dev >= 64 || !configured[dev]) {
-        e = cudaFuncSetAttribute(cawn_scan_kernel<T, W, KIND, VEC, MINB, DYN, EAR>,
-                                 cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-        if (dev >= 0 && dev < 64) configured[dev] = true;
-    }
-    // Launched with programmatic stream serialisation: when the launch before it on the stream
-    // is one of these kernels, this one may start occupying SMs while that one drains; the
-    // kernel itself waits for its predecessor before touching anything that one may have written.
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)sp.G, (unsigned)sp.B, (unsigned)sp.K);
-    cfg.blockDim = dim3(W * 32, 1, 1);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, cawn_scan_kernel<T, W, KIND, VEC, MINB, DYN, EAR>, sp);
-}
-template <int T, int W, int KIND, int MINB, bool DYN = false, bool EAR = false>
-cudaError_t launch_scan(const ScanParams &sp, cudaStream_t st)
-{
-    return sp.C % 2 == 0 ? launch_scan_inst<T, W, KIND, true, MINB, DYN, EAR>(sp, st)
-                         : launch_scan_inst<T, W, KIND, false, MINB, DYN, EAR>(sp, st);
 }
 
 // First-wave stagger of the static forward scan: about two thirds of the time one SM's share of
@@ -162,36 +124,26 @@ void set_stagger(ScanParams &sp, TileShape ts)
     sp.stagger_slots = 3;
 }
 
-inline cudaError_t launch_fwd(TileShape ts, const ScanParams &sp, cudaStream_t st, bool dyn = false)
+constexpr uint32_t kBf16Flags = CAWN_FLAG_INPUT_BF16 | CAWN_FLAG_OUTPUT_BF16;
+inline int io_of(const cawn_params *p)
 {
-    if (sp.ear_w != nullptr) {
-        if (ts.T == 16) return launch_scan<16, 8, KIND_FWD, 3, false, true>(sp, st);
-        return launch_scan<4, 4, KIND_FWD, 8, false, true>(sp, st);
-    }
-    if (dyn) {
-        if (ts.T == 16) return launch_scan<16, 8, KIND_FWD, 2, true>(sp, st);
-        return launch_scan<4, 4, KIND_FWD, 8, true>(sp, st);
-    }
-    if (ts.T == 16) return launch_scan<16, 8, KIND_FWD, 3>(sp, st);
-    return launch_scan<4, 4, KIND_FWD, 8>(sp, st);
+    return ((p->flags & CAWN_FLAG_INPUT_BF16) ? IO_IN_BF16 : 0) | ((p->flags & CAWN_FLAG_OUTPUT_BF16) ? IO_OUT_BF16 : 0);
 }
-inline cudaError_t launch_fused(TileShape ts, const ScanParams &sp, cudaStream_t st)
+
+inline cudaError_t launch_fwd(TileShape ts, const ScanParams &sp, cudaStream_t st, bool dyn = false, int io = 0)
 {
-    if (sp.ear_w != nullptr) {
-        if (ts.T == 16) return launch_scan<16, 8, KIND_FUSED, 3, false, true>(sp, st);
-        return launch_scan<4, 4, KIND_FUSED, 8, false, true>(sp, st);
-    }
-    if (ts.T == 16) return launch_scan<16, 8, KIND_FUSED, 3>(sp, st);
-    return launch_scan<4, 4, KIND_FUSED, 8>(sp, st);
+    if (io != 0) return launch_fwd_bf16(ts, sp, st, io);
+    if (sp.ear_w != nullptr) return launch_fwd_ear(ts, sp, st);
+    return dyn ? launch_fwd_dynamic(ts, sp, st) : launch_fwd_static(ts, sp, st);
+}
+inline cudaError_t launch_fused(TileShape ts, const ScanParams &sp, cudaStream_t st, int io = 0)
+{
+    if (io != 0) return launch_fused_bf16(ts, sp, st, io);
+    return sp.ear_w != nullptr ? launch_fused_ear(ts, sp, st) : launch_fused_plain(ts, sp, st);
 }
 inline cudaError_t launch_bwd(TileShape ts, const ScanParams &sp, cudaStream_t st, bool dyn = false)
 {
-    if (dyn) {
-        if (ts.T == 8) return launch_scan<8, 8, KIND_BWD, 2, true>(sp, st);
-        return launch_scan<4, 4, KIND_BWD, 8, true>(sp, st);
-    }
-    if (ts.T == 8) return launch_scan<8, 8, KIND_BWD, 3>(sp, st);
-    return launch_scan<4, 4, KIND_BWD, 8>(sp, st);
+    return dyn ? launch_bwd_dynamic(ts, sp, st) : launch_bwd_static(ts, sp, st);
 }
 
 // Host-staged forward: layout of the device scratch.
@@ -325,6 +277,8 @@ static int fwd_common(const cawn_params *params, const void *input,
     if (rc != CAWN_OK) return rc;
     const bool dyn = (params->flags & CAWN_FLAG_RETENTION_DYNAMIC) != 0;
     const bool fused = params->conv_k != 0;
+    const int io = io_of(params);
+    if (io != 0 && (dyn || ear_w != nullptr)) return CAWN_ERR_UNSUPPORTED;
     if (ear_w != nullptr) {
         if (ear_k != 1 && ear_k != 3) return CAWN_ERR_UNSUPPORTED;
         if (dyn) return CAWN_ERR_UNSUPPORTED;
@@ -394,13 +348,13 @@ static int fwd_common(const cawn_params *params, const void *input,
             sp.tail_in = state_in ? reinterpret_cast<const float *>(reinterpret_cast<const char *>(state_in) + tail_off) : nullptr;
             sp.tail_out = state_out ? reinterpret_cast<float *>(reinterpret_cast<char *>(state_out) + tail_off) : nullptr;
         }
-        if (launch_fused(ts, sp, st) != cudaSuccess) return CAWN_ERR_CUDA;
+        if (launch_fused(ts, sp, st, io) != cudaSuccess) return CAWN_ERR_CUDA;
         return CAWN_OK;
     }
     sp.gamma_logit = gamma_logit; sp.freq_bias = freq_bias; sp.H = params->H; sp.F = params->F;
     sp.early_loads = (params->flags & CAWN_FLAG_INPUT_INDEPENDENT) ? 1 : 0;
-    if (!dyn && ts.T == 16) set_stagger(sp, ts);
-    if (launch_fwd(ts, sp, st, dyn) != cudaSuccess) return CAWN_ERR_CUDA;
+    if (!dyn && ts.T == 16 && io == 0) set_stagger(sp, ts);
+    if (launch_fwd(ts, sp, st, dyn, io) != cudaSuccess) return CAWN_ERR_CUDA;
     return CAWN_OK;
 }
 
@@ -441,6 +395,7 @@ static int bwd_common(const cawn_params *params, bool dyn, const void *saved, in
 {
     int rc = check_params(params);
     if (rc != CAWN_OK) return rc;
+    if (params->flags & kBf16Flags) return CAWN_ERR_UNSUPPORTED;   // fp32 storage only here
     if (params->conv_k != 0) return CAWN_ERR_UNSUPPORTED;
     if (saved_kind != CAWN_SAVED_STATES && saved_kind != CAWN_SAVED_PUSHES) return CAWN_ERR_INVALID_ARG;
     if (theta == nullptr || workspace == nullptr) return CAWN_ERR_NULL_POINTER;
@@ -574,6 +529,7 @@ int cawn_mixing_bwd(const cawn_params *params, const float *h, const float *conv
 {
     int rc = check_params(params);
     if (rc != CAWN_OK) return rc;
+    if (params->flags & kBf16Flags) return CAWN_ERR_UNSUPPORTED;   // fp32 storage only here
     if (params->conv_k < 1 || params->conv_k > 4 || (params->flags & CAWN_FLAG_RETENTION_DYNAMIC))
         return CAWN_ERR_UNSUPPORTED;
     if ((params->flags & CAWN_FLAG_PRELUDE_CLAMP_SILU) && params->gate_eps > 0.4f) return CAWN_ERR_UNSUPPORTED;
@@ -690,6 +646,7 @@ int cawn_phase_accumulate_fwd_host(const cawn_params *params, const void *p_host
 {
     int rc = check_params(params);
     if (rc != CAWN_OK) return rc;
+    if (params->flags & kBf16Flags) return CAWN_ERR_UNSUPPORTED;   // fp32 storage only here
     if (params->conv_k != 0 || (params->flags & CAWN_FLAG_RETENTION_DYNAMIC))
         return CAWN_ERR_UNSUPPORTED;
     if (!gamma_host || !theta_host || !device_scratch) return CAWN_ERR_NULL_POINTER;

@@ -1,0 +1,11 @@
+#include "cawn_launch_impl.cuh"
+
+namespace cawn {
+
+cudaError_t launch_fwd_ear(TileShape ts, const ScanParams &sp, cudaStream_t st)
+{
+    if (ts.T == 16) return launch_scan<16, 8, KIND_FWD, 3, false, true>(sp, st);
+    return launch_scan<4, 4, KIND_FWD, 8, false, true>(sp, st);
+}
+
+}  // namespace cawn

@@ -37,11 +37,27 @@
 // accumulates sum conj(lam_t) P_{t-1} per channel for the retention and rotation gradients.
 #pragma once
 #include "cawn_device.cuh"
+#include <cuda_bf16.h>
 #include <type_traits>
 
 namespace cawn {
 
 enum : int { KIND_FWD = 0, KIND_FUSED = 1, KIND_BWD = 2 };
+
+// Storage type of the forward's input (pushes or hidden rows) and output; the arithmetic and the
+// carried state are fp32 either way.
+enum : int { IO_F32 = 0, IO_IN_BF16 = 1, IO_OUT_BF16 = 2 };
+
+// A bf16 is the upper half of a float: widening is exact.
+__device__ __forceinline__ float2 bf16x2_to_float2(unsigned u)
+{
+    return make_float2(__uint_as_float(u << 16), __uint_as_float(u & 0xffff0000u));
+}
+__device__ __forceinline__ unsigned float2_to_bf16x2(float lo, float hi)
+{
+    const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);       // round to nearest even
+    return *reinterpret_cast<const unsigned *>(&v);
+}
 
 // Rows of hidden-state history in front of a tile that the fused conv prelude may read.
 constexpr int kHalo = 3;
@@ -52,6 +68,7 @@ constexpr int kWindow = 7;
 struct ScanParams {
     const void *in;              // FWD: pushes p;  BWD: grad_y              [B,L,C] complex64
                                  // FUSED: hidden states h                   [B,L,C] float
+                                 // (IO_IN_BF16: pairs of bf16 / bf16; IO_OUT_BF16: y as pairs of bf16)
     void *out;                   // FWD: y;         BWD: grad_p
     const void *aux;             // BWD: saved unclamped states P (NULL: no parameter sums)
     const float *gamma, *theta;  // [C]
@@ -130,6 +147,11 @@ __device__ __forceinline__ void cp_async8(uint32_t dst, const void *src)
 {
     asm volatile("cp.async.ca.shared.global [%0+%2], [%1], 8;" :: "r"(dst), "l"(src), "n"(OFF) : "memory");
 }
+template <int OFF>
+__device__ __forceinline__ void cp_async4o(uint32_t dst, const void *src)
+{
+    asm volatile("cp.async.ca.shared.global [%0+%2], [%1], 4;" :: "r"(dst), "l"(src), "n"(OFF) : "memory");
+}
 __device__ __forceinline__ void cp_async4(uint32_t dst, const void *src)
 {
     asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" :: "r"(dst), "l"(src) : "memory");
@@ -163,11 +185,21 @@ __device__ __forceinline__ const char *row_ptr(const char *base, int step, int i
 
 // Copy (asynchronously) or zero one row piece of this lane: two adjacent complex64 at byte
 // offset OFF from the thread's first piece (`dst` generic, `dst_s` the same in shared space).
-template <bool VEC, int OFF>
+// HALF: the source holds two complex bf16 (8 bytes); they land in the first half of the piece and
+// are widened in place by the thread that owns it.
+template <bool VEC, int OFF, bool HALF = false>
 __device__ __forceinline__ void fetch_piece(float4 *dst, uint32_t dst_s, const char *src, bool vA, bool vB)
 {
     float4 *d4 = reinterpret_cast<float4 *>(reinterpret_cast<char *>(dst) + OFF);
-    if (VEC) {
+    if constexpr (HALF) {
+        unsigned *d = reinterpret_cast<unsigned *>(d4);
+        if (VEC) {
+            if (vA) cp_async8<OFF>(dst_s, src); else { d[0] = 0u; d[1] = 0u; }
+        } else {
+            if (vA) cp_async4o<OFF>(dst_s, src); else d[0] = 0u;
+            if (vB) cp_async4o<OFF + 4>(dst_s, src + 4); else d[1] = 0u;
+        }
+    } else if (VEC) {
         if (vA) cp_async16<OFF>(dst_s, src); else *d4 = zero4();
     } else {
         float2 *d = reinterpret_cast<float2 *>(d4);
@@ -179,24 +211,26 @@ __device__ __forceinline__ void fetch_piece(float4 *dst, uint32_t dst_s, const c
 // Unrolled helper: issue the T copies of one thread (rows i = 0..T-1, `step` bytes apart in
 // global memory, 512 bytes apart in shared memory), committing one copy group per GR rows
 // (GR = 0: the caller commits).  valid(i) says whether row i exists.
-template <bool VEC, int T, int GR, int I = 0, typename F>
+template <bool VEC, int T, int GR, int I = 0, bool HALF = false, typename F>
 __device__ __forceinline__ void fetch_rows(float4 *dst, uint32_t dst_s, const char *src, int step,
                                            bool vA, bool vB, F valid)
 {
     if constexpr (I < T) {
         const bool row = valid(I);
-        fetch_piece<VEC, I * 512>(dst, dst_s, row_ptr(src, step, I), row && vA, row && vB);
+        fetch_piece<VEC, I * 512, HALF>(dst, dst_s, row_ptr(src, step, I), row && vA, row && vB);
         if constexpr (GR > 0 && (I + 1) % GR == 0) cp_async_commit();
-        fetch_rows<VEC, T, GR, I + 1>(dst, dst_s, src, step, vA, vB, valid);
+        fetch_rows<VEC, T, GR, I + 1, HALF>(dst, dst_s, src, step, vA, vB, valid);
     }
 }
 
-template <int T, int W, int KIND, bool VEC, bool DYN, bool FULL, bool EAR = false>
+template <int T, int W, int KIND, bool VEC, bool DYN, bool FULL, bool EAR = false, int IO = IO_F32>
 __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, KIND, DYN> &sm,
                                           const int g, const int b, const int k)
 {
     static_assert(!(DYN && KIND == KIND_FUSED), "time-varying retention is not built for the fused path");
     static_assert(!(EAR && (DYN || KIND == KIND_BWD)), "the Ear epilogue belongs to the static forward");
+    static_assert(IO == IO_F32 || (!EAR && !DYN && KIND != KIND_BWD), "bf16 storage is built for the static forward");
+    constexpr bool IN16 = (IO & IO_IN_BF16) != 0, OUT16 = (IO & IO_OUT_BF16) != 0;
     constexpr bool REV = (KIND == KIND_BWD);
     constexpr int TILE = T * W;
     constexpr int M = kWindow;
@@ -243,13 +277,28 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
     float *const hs = reinterpret_cast<float *>(&sm.tile[0][0][0]) + (TILE * 128 - (TILE + kHalo) * 64);
     if constexpr (KIND == KIND_FUSED) {
         const float *hin = reinterpret_cast<const float *>(prm.in);
+        const unsigned short *hin16 = reinterpret_cast<const unsigned short *>(prm.in);
         float *mine = hs + (kHalo + w * T) * 64 + 2 * lane;
         const float *r = hin + e0;
+        const unsigned short *r16 = hin16 + e0;
+        // a bf16 hidden value is kept in its float slot as the float it widens to
+        auto widen = [](unsigned short v) -> float { return __uint_as_float((unsigned)v << 16); };
 #pragma unroll
         for (int i = 0; i < T; ++i) {
             const bool row = FULL || i < nvalid;
             float *d = mine + i * 64;
-            if (VEC) {
+            if constexpr (IN16) {
+                // the pair of bf16 goes into the first word of the slot; phase 1 widens it
+                if (VEC) {
+                    if (row && vA) cp_async4(smem_addr(d), r16); else d[0] = 0.f;
+                } else {
+                    unsigned lo = 0u, hi = 0u;
+                    if (row && vA) lo = r16[0];
+                    if (row && vB) hi = r16[1];
+                    reinterpret_cast<unsigned *>(d)[0] = lo | (hi << 16);
+                }
+                r16 += C;
+            } else if (VEC) {
                 if (row && vA) cp_async8<0>(smem_addr(d), r); else *reinterpret_cast<float2 *>(d) = make_float2(0.f, 0.f);
             } else {
                 if (row && vA) cp_async4(smem_addr(d), r); else d[0] = 0.f;
@@ -272,14 +321,28 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
                     if (t >= 0) src = hin + ((long long)b * L + t) * C + c0;
                     else if (prm.tail_in != nullptr) src = prm.tail_in + ((long long)b * Kh + (Kh + t)) * C + c0;
                 }
+                if constexpr (IN16) {
+                    // earlier rows of h are bf16 (widened here, stored as floats like the carried
+                    // tail, which is fp32 in the state blob)
+                    if (j >= kHalo - Kh && t >= 0) {
+                        const unsigned short *s16 = hin16 + ((long long)b * L + t) * C + c0;
+                        d[0] = vA ? widen(s16[0]) : 0.f;
+                        d[1] = vB ? widen(s16[1]) : 0.f;
+                        continue;
+                    }
+                }
                 if (src != nullptr && vA) cp_async4(smem_addr(d), src); else d[0] = 0.f;
                 if (src != nullptr && vB) cp_async4(smem_addr(d + 1), src + 1); else d[1] = 0.f;
             }
         }
         cp_async_commit();
     } else {
-        fetch_rows<VEC, T, GR>(xs, smem_addr(xs), reinterpret_cast<const char *>(prm.in) + e0 * 8, rowbytes, vA, vB,
-                               [&](int i) { return FULL || i < nvalid; });
+        if constexpr (IN16)
+            fetch_rows<VEC, T, GR, 0, true>(xs, smem_addr(xs), reinterpret_cast<const char *>(prm.in) + e0 * 4, rowbytes / 2,
+                                            vA, vB, [&](int i) { return FULL || i < nvalid; });
+        else
+            fetch_rows<VEC, T, GR>(xs, smem_addr(xs), reinterpret_cast<const char *>(prm.in) + e0 * 8, rowbytes, vA, vB,
+                                   [&](int i) { return FULL || i < nvalid; });
     }
     if constexpr (KIND == KIND_BWD) {
         float4 *const qs = &sm.tile[1][w * T][lane];
@@ -400,8 +463,13 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
         // magnitude sigmoid(x), phase pi*tanh(x), gate on the conv output, push m (cos, sin).
         float2 hv[T + kHalo];
 #pragma unroll
-        for (int r = 0; r < T + kHalo; ++r)
-            hv[r] = *reinterpret_cast<const float2 *>(hs + (w * T + r) * 64 + 2 * lane);
+        for (int r = 0; r < T + kHalo; ++r) {
+            const float *slot = hs + (w * T + r) * 64 + 2 * lane;
+            // own rows of a bf16 input are still packed pairs; history rows (r < kHalo as seen
+            // from warp 0, other warps' rows otherwise) follow the same rule row by row
+            if (IN16 && (w * T + r) >= kHalo) hv[r] = bf16x2_to_float2(*reinterpret_cast<const unsigned *>(slot));
+            else hv[r] = *reinterpret_cast<const float2 *>(slot);
+        }
         if (early_ptr != nullptr) {
             er0 = ld_record(early_ptr + 2 * lane);
             er1 = ld_record(early_ptr + 2 * lane + 1);
@@ -507,7 +575,14 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
                         er1 = ld_record(early_ptr + 2 * lane + 1);
                     }
                 }
-                float4 v = xs[i * 32];
+                float4 v;
+                if (IN16 && !EXACT) {                     // first touch: widen the staged bf16 in place
+                    const uint2 u = *reinterpret_cast<const uint2 *>(&xs[i * 32]);
+                    const float2 cA = bf16x2_to_float2(u.x), cB = bf16x2_to_float2(u.y);
+                    v = make_float4(cA.x, cA.y, cB.x, cB.y);
+                } else {
+                    v = xs[i * 32];
+                }
                 bool oA, oB;
                 if (EXACT) {
                     oA = ((double)v.x * (double)v.x + (double)v.y * (double)v.y >= prm.eps2);
@@ -658,7 +733,8 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
 
         // EAR: a planar row is 2C floats, as long as an interleaved one; the real parts of this
         // lane's two channels sit c0 floats into it, the imaginary parts C floats further
-        char *const rbase = reinterpret_cast<char *>(prm.out) + (EAR ? (e0 - c0) * 8 + c0 * 4 : e0 * 8);
+        char *const rbase = reinterpret_cast<char *>(prm.out) + (EAR ? (e0 - c0) * 8 + c0 * 4 : (OUT16 ? e0 * 4 : e0 * 8));
+        const int orow = OUT16 ? rowbytes / 2 : rowbytes;
         const float cl = prm.clampv;
         // Ear taps of this lane's two channels, real and imaginary part: (left, centre, right,
         // bias).  A tap whose source harmonic lies outside the head is zero (zero padding), so the
@@ -686,8 +762,16 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
         // one output row of this lane's channel pair; every lane of the warp takes part (the Ear
         // form exchanges edge channels with the neighbouring lanes)
         auto store_row = [&](int i, float4 o) {
-            char *r = const_cast<char *>(row_ptr(rbase, rowbytes, i));
-            if constexpr (EAR) {
+            char *r = const_cast<char *>(row_ptr(rbase, orow, i));
+            if constexpr (OUT16) {
+                const unsigned pA = float2_to_bf16x2(o.x, o.y), pB = float2_to_bf16x2(o.z, o.w);
+                if (VEC) {
+                    if (vA) __stcs(reinterpret_cast<uint2 *>(r), make_uint2(pA, pB));
+                } else {
+                    if (vA) __stcs(reinterpret_cast<unsigned *>(r), pA);
+                    if (vB) __stcs(reinterpret_cast<unsigned *>(r) + 1, pB);
+                }
+            } else if constexpr (EAR) {
                 const float lre = __shfl_up_sync(0xffffffffu, o.z, 1), lim = __shfl_up_sync(0xffffffffu, o.w, 1);
                 const float rre = __shfl_down_sync(0xffffffffu, o.x, 1), rim = __shfl_down_sync(0xffffffffu, o.y, 1);
                 const float zrA = fmaf(ewr[0][0], lre, fmaf(ewr[0][1], o.x, fmaf(ewr[0][2], o.z, ewr[0][3])));
@@ -810,7 +894,11 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
             for (int r = 0; r < Kh; ++r) {
                 const long long t = L - Kh + r;
                 float vA_ = 0.f, vB_ = 0.f;
-                if (t >= 0) {
+                if (t >= 0 && IN16) {
+                    const unsigned short *src = reinterpret_cast<const unsigned short *>(prm.in) + ((long long)b * L + t) * C + c0;
+                    if (vA) vA_ = __uint_as_float((unsigned)src[0] << 16);
+                    if (vB) vB_ = __uint_as_float((unsigned)src[1] << 16);
+                } else if (t >= 0) {
                     const float *src = hin + ((long long)b * L + t) * C + c0;
                     if (vA) vA_ = src[0];
                     if (vB) vB_ = src[1];
@@ -859,7 +947,7 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
     }
 }
 
-template <int T, int W, int KIND, bool VEC, int MINB, bool DYN = false, bool EAR = false>
+template <int T, int W, int KIND, bool VEC, int MINB, bool DYN = false, bool EAR = false, int IO = IO_F32>
 __global__ void __launch_bounds__(W * 32, MINB) cawn_scan_kernel(const ScanParams prm)
 {
     constexpr int TILE = T * W;
@@ -872,79 +960,8 @@ __global__ void __launch_bounds__(W * 32, MINB) cawn_scan_kernel(const ScanParam
     const int k = blockIdx.z;                         // tile index along (logical) time
     grid_launch_dependents();
     const bool full = ((long long)(k + 1) * TILE <= prm.L) && (g * 64 + 64 <= prm.C);
-    if (full) scan_tile<T, W, KIND, VEC, DYN, true, EAR>(prm, sm, g, b, k);
-    else      scan_tile<T, W, KIND, VEC, DYN, false, EAR>(prm, sm, g, b, k);
-}
-
-// grad_gamma_j = Re(e^{i theta} Q_j), grad_theta_j = -Im(a_j Q_j), Q_j = sum of the per-tile
-// partials in a fixed order, in double.  One warp per channel.
-__global__ void cawn_bwd_finalize_kernel(const float2 *qpart, int nparts, int C,
-                                         const float *gamma, const float *theta,
-                                         float *grad_gamma, float *grad_theta, float clampv)
-{
-    const int lane = threadIdx.x & 31;
-    const int ch = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    if (ch >= C) return;
-    double sr = 0.0, si = 0.0;
-    for (int p = lane; p < nparts; p += 32) {
-        const float2 q = qpart[(long long)p * C + ch];
-        sr += (double)q.x;
-        si += (double)q.y;
-    }
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) {
-        sr += __shfl_down_sync(0xffffffffu, sr, off);
-        si += __shfl_down_sync(0xffffffffu, si, off);
-    }
-    if (lane == 0) {
-        const double gm = gamma != nullptr ? (double)gamma[ch] : 1.0;   // time-varying: already in Q
-        double sn, cs;
-        sincos((double)theta[ch], &sn, &cs);
-        double dg = cs * sr - sn * si;
-        const double dth = -gm * (cs * si + sn * sr);
-        if (clampv > 0.f) dg = fmin(fmax(dg, -(double)clampv), (double)clampv);
-        if (grad_gamma != nullptr) grad_gamma[ch] = (float)dg;
-        if (grad_theta != nullptr) grad_theta[ch] = (float)dth;
-    }
-}
-
-// Time-varying retention: grad_freq_bias[k] = sum over tiles and heads of the per-channel
-// partial sums of the logit gradient, in a fixed order, in double.  One warp per harmonic.
-__global__ void cawn_bwd_freq_bias_kernel(const float *spart, int nparts, int H, int F, float *grad_freq_bias)
-{
-    const int lane = threadIdx.x & 31;
-    const int kf = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    if (kf >= F) return;
-    const long long C = (long long)H * F;
-    double acc = 0.0;
-    for (long long i = lane; i < (long long)nparts * H; i += 32) {
-        const long long part = i / H, h = i % H;
-        acc += (double)spart[part * C + h * F + kf];
-    }
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) acc += __shfl_down_sync(0xffffffffu, acc, off);
-    if (lane == 0) grad_freq_bias[kf] = (float)acc;
-}
-
-// state_out = a^n * state_prev + state_local with a^n = gamma^n (cos n theta, sin n theta)
-// evaluated in double.
-__global__ void cawn_state_carry_kernel(const float2 *prev, const float2 *local, float2 *out,
-                                        const float *gamma, const float *theta,
-                                        long long n_steps, int B, int C)
-{
-    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    if (idx >= (long long)B * C) return;
-    const int ch = (int)(idx % C);
-    const double gm = (double)gamma[ch], th = (double)theta[ch];
-    const double mag = pow(gm, (double)n_steps);
-    double sn, cs;
-    sincos(th * (double)n_steps, &sn, &cs);
-    const float2 p = prev[idx], l = local[idx];
-    const double pr = (double)p.x, pi = (double)p.y;
-    float2 o;
-    o.x = (float)((double)l.x + mag * (pr * cs - pi * sn));
-    o.y = (float)((double)l.y + mag * (pr * sn + pi * cs));
-    out[idx] = o;
+    if (full) scan_tile<T, W, KIND, VEC, DYN, true, EAR, IO>(prm, sm, g, b, k);
+    else      scan_tile<T, W, KIND, VEC, DYN, false, EAR, IO>(prm, sm, g, b, k);
 }
 
 }  // namespace cawn

@@ -154,3 +154,23 @@ def gate_tau(gate_eps: float) -> np.float32:
     if gate_eps >= 1.0:
         return np.float32(np.inf)
     return np.float32(math.log(gate_eps / (1.0 - gate_eps)))
+
+
+def to_bf16(a):
+    """Round a float array to bfloat16 (nearest even).  Returns (bits uint16, the same values widened
+    back to float32); complex input is treated as (re, im) pairs.  Storage conversion only: the
+    bf16-input parity cases feed the bits to the device and the widened values to the oracle."""
+    a = np.ascontiguousarray(a)
+    cplx = np.iscomplexobj(a)
+    f = a.astype(np.complex64).view(np.float32) if cplx else a.astype(np.float32)
+    u = f.view(np.uint32).astype(np.uint64)
+    r = ((u + 0x7FFF + ((u >> 16) & 1)) >> 16).astype(np.uint16)
+    wide = (r.astype(np.uint32) << 16).view(np.float32)
+    if cplx:
+        return r.reshape(a.shape + (2,)), wide.view(np.complex64).reshape(a.shape)
+    return r.reshape(a.shape), wide.reshape(a.shape)
+
+
+def from_bf16(bits):
+    """bfloat16 bits (uint16) -> float32; a trailing axis of 2 is NOT folded into complex here."""
+    return (np.ascontiguousarray(bits).astype(np.uint32) << 16).view(np.float32)
