@@ -215,7 +215,8 @@ CAWN_API int cawn_phase_accumulate_bwd_dynamic(const cawn_params *params,
 
 /*
  * Backward of the fused Resonance mixing path (cawn_phase_accumulate_fwd with conv_k >= 1,
- * static retention): reverse scan, then the prelude's chain rule.
+ * static retention): the reverse scan with the prelude's chain rule as its epilogue, one pass
+ * over grad_y, the saved states and h.
  *   lam   = reverse scan of grad_y (as cawn_phase_accumulate_bwd); it is the gradient of the pushes
  *   magnitude m = sigmoid(x), phase ph = pi tanh(x), push z = m_used (cos ph, sin ph):
  *     d m  = Re(conj(lam) e^{i ph})                    straight-through: flows open or closed
@@ -231,8 +232,8 @@ CAWN_API int cawn_phase_accumulate_bwd_dynamic(const cawn_params *params,
  *               and conv-history part, e.g. the next chunk's grad_state_in) or NULL.
  * grad_h [B,L,C] float; grad_conv_w [C,conv_k], grad_conv_bias [C], grad_gamma [C], grad_theta [C]
  *               float or NULL; grad_state_in: state blob of gradients or NULL.  All device.
- * workspace:    >= cawn_workspace_bytes(CAWN_OP_MIXING_BWD), initialised once; it also holds the
- *               push gradient lam (B*L*C complex64) between the two kernels.
+ * workspace:    >= cawn_workspace_bytes(CAWN_OP_MIXING_BWD), initialised once (carry records, per-tile
+ *               partial sums, and the few rows exchanged at tile seams; O(B*C*L/64)).
  * Deterministic (parameter sums: per-CTA partials combined in a fixed order in double).
  */
 CAWN_API int cawn_mixing_bwd(const cawn_params *params,

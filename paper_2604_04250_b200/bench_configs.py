@@ -222,9 +222,9 @@ def _cfg4_bwd(args, cb, inputs, dev):
                                             grad_conv_bias=gb, grad_gamma=gg, grad_theta=gt),
                max(args.steps // 2, 5), args.warmup)
     assert cb.cawn_poll_status(wb) == 0
-    # reads grad_y (8) + P (8) + h (4), writes grad_h (4); lambda (8 written + 8 read) is internal traffic
+    # reads grad_y (8) + P (8) + h (4), writes grad_h (4)
     _report("cfg4_mixing_bwd" if B == cfg.B else "cfg4_mixing_bwd_B%d" % B, B * L, B * L * C * 24, ms, 4,
-            {"note": "algorithmic bytes exclude the workspace pass of the adjoint states (16 B/elem more)"})
+            {"note": "reverse scan with the prelude backward as its epilogue, seam rows, two reductions"})
 
 
 def _cfg2(args, cb, inputs, dev, IND):

@@ -2,7 +2,6 @@
 #include "../../include/cawn.h"
 #include "cawn_launch.cuh"
 #include "cawn_small_kernels.cuh"
-#include "cawn_prelude_bwd.cuh"
 
 #include <math.h>
 #include <string.h>
@@ -146,6 +145,25 @@ inline cudaError_t launch_bwd(TileShape ts, const ScanParams &sp, cudaStream_t s
     return dyn ? launch_bwd_dynamic(ts, sp, st) : launch_bwd_static(ts, sp, st);
 }
 
+// Workspace of cawn_mixing_bwd: header, carry records, per-tile sums for grad_gamma / grad_theta,
+// du at the tile seams, per-tile sums for the conv gradients.
+struct MixBwdLayout {
+    size_t off_rec, off_qpart, off_edge, off_cpart, total;
+};
+MixBwdLayout mix_bwd_layout(const cawn_params *p)
+{
+    const Geometry g = geometry(p, bwd_shape(p->L));
+    const size_t tiles = (size_t)p->B * g.K;
+    MixBwdLayout m;
+    size_t o = sizeof(WsHeader);
+    m.off_rec = o;    o += round_up(g.rec_bytes, 256);
+    m.off_qpart = o;  o += round_up(tiles * g.C * sizeof(float2), 256);
+    m.off_edge = o;   o += round_up(tiles * 6 * g.C * sizeof(float), 256);
+    m.off_cpart = o;  o += round_up(tiles * g.C * 5 * sizeof(float), 256);
+    m.total = o;
+    return m;
+}
+
 // Host-staged forward: layout of the device scratch.
 struct HostStage {
     size_t off_x, off_gamma, off_theta, off_state, off_mask, off_ws, total;
@@ -231,18 +249,9 @@ int cawn_workspace_bytes(const cawn_params *params, int op, size_t *bytes)
         *bytes = total;
         return CAWN_OK;
     }
-    case CAWN_OP_MIXING_BWD: {
-        cawn_params q = *params;
-        q.conv_k = 0;                                   // the scan part is the Cartesian backward
-        size_t scan = 0;
-        const int rc2 = cawn_workspace_bytes(&q, CAWN_OP_BWD_SAVED, &scan);
-        if (rc2 != CAWN_OK) return rc2;
-        const int64_t rows_per_cta = (int64_t)kPbRows * kPbWarps;
-        const size_t rt = (size_t)((params->L + rows_per_cta - 1) / rows_per_cta);
-        *bytes = round_up(scan, 256) + round_up(n * sizeof(float2), 256) +
-                 round_up((size_t)params->B * (rt ? rt : 1) * (size_t)params->H * params->F * 5 * sizeof(float), 256);
+    case CAWN_OP_MIXING_BWD:
+        *bytes = mix_bwd_layout(params).total;
         return CAWN_OK;
-    }
     case CAWN_OP_STATE:
         *bytes = state_blob_bytes(params);
         return CAWN_OK;
@@ -538,67 +547,88 @@ int cawn_mixing_bwd(const cawn_params *params, const float *h, const float *conv
     if (!aligned(h, 16) || !aligned(grad_h, 16) || !aligned(workspace, 16) || !aligned(state_in, 16) ||
         !aligned(grad_state_out, 16) || !aligned(grad_state_in, 16))
         return CAWN_ERR_MISALIGNED;
-    size_t need = 0;
-    rc = cawn_workspace_bytes(params, CAWN_OP_MIXING_BWD, &need);
-    if (rc != CAWN_OK) return rc;
-    if (workspace_bytes < need) return CAWN_ERR_WORKSPACE_TOO_SMALL;
+    const MixBwdLayout lay = mix_bwd_layout(params);
+    if (workspace_bytes < lay.total) return CAWN_ERR_WORKSPACE_TOO_SMALL;
+    const TileShape ts = bwd_shape(params->L);
+    const Geometry g = geometry(params, ts);
+    if (!grid_ok(params, g) || g.K + 1 > 65535) return CAWN_ERR_UNSUPPORTED;
     cudaStream_t st = (cudaStream_t)cuda_stream;
-    const int C = params->H * params->F, Kc = params->conv_k, Kh = Kc - 1;
-    const size_t n = (size_t)params->B * (size_t)params->L * C;
+    const int C = g.C, Kc = params->conv_k, Kh = Kc - 1;
     const size_t tail_off = round_up((size_t)params->B * C * sizeof(float2), 16);
+    const bool want_scan_param = grad_gamma != nullptr || grad_theta != nullptr;
+    const bool want_conv_param = grad_conv_w != nullptr || grad_conv_bias != nullptr;
+    if (params->L > 0 && want_scan_param && saved_states == nullptr) return CAWN_ERR_NULL_POINTER;
+    if (!aligned(saved_states, 16) || !aligned(grad_y, 16)) return CAWN_ERR_MISALIGNED;
 
-    // 1. reverse scan: lam into the workspace, grad_gamma / grad_theta / the state part of grad_state_in
-    cawn_params q = *params;
-    q.conv_k = 0;
-    size_t scan_bytes = 0;
-    rc = cawn_workspace_bytes(&q, CAWN_OP_BWD_SAVED, &scan_bytes);
-    if (rc != CAWN_OK) return rc;
-    char *base = reinterpret_cast<char *>(workspace);
-    float2 *lam = reinterpret_cast<float2 *>(base + round_up(scan_bytes, 256));
-    float *part = reinterpret_cast<float *>(base + round_up(scan_bytes, 256) + round_up(n * sizeof(float2), 256));
-    rc = bwd_common(&q, false, saved_states, CAWN_SAVED_STATES, gamma, nullptr, nullptr, theta, state_in, grad_y,
-                    grad_state_out, lam, grad_gamma, nullptr, nullptr, grad_theta, grad_state_in,
-                    workspace, scan_bytes, st);
-    if (rc != CAWN_OK) return rc;
-
-    // 2. the prelude's chain rule
-    const int64_t rows_per_cta = (int64_t)kPbRows * kPbWarps;
-    const int RT = (int)((params->L + rows_per_cta - 1) / rows_per_cta);
-    if (params->L > 0) {
-        if (RT > 65535 || params->B > 65535) return CAWN_ERR_UNSUPPORTED;
-        PreludeBwdParams pp;
-        memset(&pp, 0, sizeof(pp));
-        pp.h = h; pp.lam = lam; pp.conv_w = conv_w; pp.conv_bias = conv_bias;
-        if (Kh > 0) {
-            pp.tail_in = state_in ? reinterpret_cast<const float *>(reinterpret_cast<const char *>(state_in) + tail_off) : nullptr;
-            pp.dtail_out = grad_state_out ? reinterpret_cast<const float *>(reinterpret_cast<const char *>(grad_state_out) + tail_off) : nullptr;
-            pp.dtail_in = grad_state_in ? reinterpret_cast<float *>(reinterpret_cast<char *>(grad_state_in) + tail_off) : nullptr;
-        }
-        pp.dh = grad_h; pp.part = part;
-        pp.L = params->L; pp.B = params->B; pp.C = C; pp.G = (C + 63) / 64; pp.RT = RT; pp.Kc = Kc;
-        pp.clamp_silu = (params->flags & CAWN_FLAG_PRELUDE_CLAMP_SILU) ? 1 : 0;
-        pp.gate_tau = params->gate_tau;
-        const dim3 grid((unsigned)pp.G, (unsigned)params->B, (unsigned)RT);
-        if (C % 2 == 0) cawn_prelude_bwd_kernel<true><<<grid, kPbWarps * 32, 0, st>>>(pp);
-        else            cawn_prelude_bwd_kernel<false><<<grid, kPbWarps * 32, 0, st>>>(pp);
-        if (cudaGetLastError() != cudaSuccess) return CAWN_ERR_CUDA;
-        if (grad_conv_w != nullptr || grad_conv_bias != nullptr) {
-            const int warps = 8;
-            cawn_prelude_bwd_finalize_kernel<<<(C + warps - 1) / warps, warps * 32, 0, st>>>(
-                part, params->B * RT, C, Kc, grad_conv_w, grad_conv_bias);
-            if (cudaGetLastError() != cudaSuccess) return CAWN_ERR_CUDA;
-        }
-    } else {
-        // nothing ran: the incoming history gradient passes through, the parameter gradients are zero
-        if (grad_conv_w && cudaMemsetAsync(grad_conv_w, 0, (size_t)C * Kc * sizeof(float), st) != cudaSuccess) return CAWN_ERR_CUDA;
-        if (grad_conv_bias && cudaMemsetAsync(grad_conv_bias, 0, (size_t)C * sizeof(float), st) != cudaSuccess) return CAWN_ERR_CUDA;
-        if (grad_state_in != nullptr && Kh > 0) {
-            char *dst = reinterpret_cast<char *>(grad_state_in) + tail_off;
-            const size_t nb = (size_t)params->B * Kh * C * sizeof(float);
-            cudaError_t e = grad_state_out ? cudaMemcpyAsync(dst, reinterpret_cast<const char *>(grad_state_out) + tail_off, nb, cudaMemcpyDeviceToDevice, st)
-                                           : cudaMemsetAsync(dst, 0, nb, st);
+    if (params->L == 0) {
+        // nothing ran: the incoming state gradient passes through, the parameter gradients are zero
+        if (grad_state_in != nullptr && grad_state_in != grad_state_out) {
+            const size_t nb = state_blob_bytes(params);
+            cudaError_t e = grad_state_out ? cudaMemcpyAsync(grad_state_in, grad_state_out, nb, cudaMemcpyDeviceToDevice, st)
+                                           : cudaMemsetAsync(grad_state_in, 0, nb, st);
             if (e != cudaSuccess) return CAWN_ERR_CUDA;
         }
+        if (grad_conv_w && cudaMemsetAsync(grad_conv_w, 0, (size_t)C * Kc * sizeof(float), st) != cudaSuccess) return CAWN_ERR_CUDA;
+        if (grad_conv_bias && cudaMemsetAsync(grad_conv_bias, 0, (size_t)C * sizeof(float), st) != cudaSuccess) return CAWN_ERR_CUDA;
+        if (grad_gamma && cudaMemsetAsync(grad_gamma, 0, (size_t)C * sizeof(float), st) != cudaSuccess) return CAWN_ERR_CUDA;
+        if (grad_theta && cudaMemsetAsync(grad_theta, 0, (size_t)C * sizeof(float), st) != cudaSuccess) return CAWN_ERR_CUDA;
+        return CAWN_OK;
+    }
+
+    char *base = reinterpret_cast<char *>(workspace);
+    float2 *qpart = reinterpret_cast<float2 *>(base + lay.off_qpart);
+    float *edge = reinterpret_cast<float *>(base + lay.off_edge);
+    float *cpart = reinterpret_cast<float *>(base + lay.off_cpart);
+    const float *tail_in = nullptr, *dtail_out = nullptr;
+    float *dtail_in = nullptr;
+    if (Kh > 0) {
+        if (state_in) tail_in = reinterpret_cast<const float *>(reinterpret_cast<const char *>(state_in) + tail_off);
+        if (grad_state_out) dtail_out = reinterpret_cast<const float *>(reinterpret_cast<const char *>(grad_state_out) + tail_off);
+        if (grad_state_in) dtail_in = reinterpret_cast<float *>(reinterpret_cast<char *>(grad_state_in) + tail_off);
+    }
+
+    // 1. reverse scan with the prelude's chain rule and the conv transpose as its epilogue
+    ScanParams sp;
+    memset(&sp, 0, sizeof(sp));
+    sp.in = grad_y; sp.out = grad_h;
+    sp.aux = want_scan_param ? saved_states : nullptr;
+    sp.gamma = gamma; sp.theta = theta;
+    sp.state_in = reinterpret_cast<const float2 *>(state_in);
+    sp.edge_in = reinterpret_cast<const float2 *>(grad_state_out);
+    sp.state_out = reinterpret_cast<float2 *>(grad_state_in);
+    sp.ws = reinterpret_cast<WsHeader *>(workspace);
+    set_records(sp, base + lay.off_rec, g);
+    sp.qpart = want_scan_param ? qpart : nullptr;
+    sp.L = params->L; sp.B = params->B;
+    sp.clampv = params->grad_clamp_abs > 0.f ? params->grad_clamp_abs : 0.f;
+    sp.poll_limit = kPollLimit;
+    sp.H = params->H; sp.F = params->F;
+    sp.hid = h; sp.conv_w = conv_w; sp.conv_bias = conv_bias; sp.tail_in = tail_in;
+    sp.conv_k = Kc;
+    sp.clamp_silu = (params->flags & CAWN_FLAG_PRELUDE_CLAMP_SILU) ? 1 : 0;
+    sp.gate_tau = params->gate_tau;
+    sp.edge_du = edge;
+    sp.cpart = want_conv_param ? cpart : nullptr;
+    if (launch_mix_bwd(ts, sp, st) != cudaSuccess) return CAWN_ERR_CUDA;
+
+    // 2. rows at the tile seams and the gradient of the carried conv history
+    {
+        const dim3 grid((unsigned)((C + 127) / 128), (unsigned)(g.K + 1), (unsigned)params->B);
+        cawn_mix_bwd_edges_kernel<<<grid, 128, 0, st>>>(edge, conv_w, dtail_out, grad_h, dtail_in, params->L, params->B,
+                                                         C, g.K, ts.T * ts.W, Kc);
+        if (cudaGetLastError() != cudaSuccess) return CAWN_ERR_CUDA;
+    }
+    // 3. parameter gradients from the per-tile partial sums
+    const int warps = 8;
+    if (want_scan_param) {
+        cawn_bwd_finalize_kernel<<<(C + warps - 1) / warps, warps * 32, 0, st>>>(
+            qpart, params->B * g.K, C, gamma, theta, grad_gamma, grad_theta, sp.clampv);
+        if (cudaGetLastError() != cudaSuccess) return CAWN_ERR_CUDA;
+    }
+    if (want_conv_param) {
+        cawn_conv_grad_finalize_kernel<<<(C + warps - 1) / warps, warps * 32, 0, st>>>(
+            cpart, params->B * g.K, C, Kc, grad_conv_w, grad_conv_bias);
+        if (cudaGetLastError() != cudaSuccess) return CAWN_ERR_CUDA;
     }
     return CAWN_OK;
 }

@@ -19,5 +19,6 @@ cudaError_t launch_fwd_bf16(TileShape ts, const ScanParams &sp, cudaStream_t st,
 cudaError_t launch_fused_bf16(TileShape ts, const ScanParams &sp, cudaStream_t st, int io);
 cudaError_t launch_bwd_static(TileShape ts, const ScanParams &sp, cudaStream_t st);    // reverse scan
 cudaError_t launch_bwd_dynamic(TileShape ts, const ScanParams &sp, cudaStream_t st);
+cudaError_t launch_mix_bwd(TileShape ts, const ScanParams &sp, cudaStream_t st);       // reverse scan + prelude backward
 
 }  // namespace cawn

@@ -42,7 +42,10 @@
 
 namespace cawn {
 
-enum : int { KIND_FWD = 0, KIND_FUSED = 1, KIND_BWD = 2 };
+// KIND_MIXBWD: the reverse scan of KIND_BWD whose push gradient is not stored but taken straight
+// through the fused path's prelude (phasor map, straight-through gate, conv) to grad_h.
+enum : int { KIND_FWD = 0, KIND_FUSED = 1, KIND_BWD = 2, KIND_MIXBWD = 3 };
+__host__ __device__ constexpr bool kind_is_bwd(int kind) { return kind == KIND_BWD || kind == KIND_MIXBWD; }
 
 // Storage type of the forward's input (pushes or hidden rows) and output; the arithmetic and the
 // carried state are fp32 either way.
@@ -96,6 +99,11 @@ struct ScanParams {
     int conv_k;                  // 1..4
     int clamp_silu;              // clamp the conv output to +-50, then SiLU
     float gate_tau;              // gate: conv output >= gate_tau (fp32 fmaf chain, tap order)
+    // backward through the fused prelude (KIND_MIXBWD): out = grad_h [B,L,C] float
+    const float *hid;            // hidden states h [B,L,C] float
+    float *edge_du;              // [B*K][6][C]: du of a tile's three last rows in time (latest first), then of
+                                 // its three first rows (earliest first); rows a tile does not have: 0
+    float *cpart;                // [B*K][C][5] per-tile sums of du*h (four right-aligned taps) and du, or NULL
     // time-varying retention (DYN): gamma_t = sigmoid(gamma_logit[b,t,h] + freq_bias[k])
     const float *gamma_logit;    // [B][L][H]
     const float *freq_bias;      // [F]
@@ -122,8 +130,10 @@ struct ScanParams {
 template <int T, int W, int KIND, bool DYN = false>
 struct ScanSmem {
     static constexpr int TILE = T * W;
-    static constexpr int NT = (KIND == KIND_BWD) ? 2 : 1;
+    static constexpr int NT = kind_is_bwd(KIND) ? 2 : 1;
     float4 tile[NT][TILE][32];
+    // MIXBWD: hidden rows in processing order (row R = physical row t_hi - R), then kHalo rows of history
+    float hrev[KIND == KIND_MIXBWD ? TILE + kHalo : 1][KIND == KIND_MIXBWD ? 64 : 1];
     float4 sE[W][32];
     float4 sR[kWindow + 1][32];
     float sCoef[64][6];
@@ -223,15 +233,46 @@ __device__ __forceinline__ void fetch_rows(float4 *dst, uint32_t dst_s, const ch
     }
 }
 
+// Chain rule of the fused prelude for one channel at one step: from the push gradient
+// (lr, li) = dLoss/d(Re z, Im z) and the conv output u to dLoss/du.  z = m_used (cos ph, sin ph)
+// with m = sigmoid(x), ph = pi tanh(x), x = u (or SiLU(clamp(u)) with `act`), m_used = m where the
+// gate is open, else 0.  Straight-through gate: the magnitude path ignores the gate
+// (dm = lr cos ph + li sin ph), the phase path is scaled by the gated magnitude.
+// m, tanh, sin and cos are recomputed exactly as the forward computes them.
+__device__ __forceinline__ float prelude_du(float u, float lr, float li, bool act, float tau)
+{
+    float x = u, dxdu = 1.f;
+    if (act) {
+        const float v = fminf(fmaxf(u, -50.f), 50.f);
+        const float sg = __fdividef(1.f, 1.f + __expf(-v));
+        x = v * sg;
+        dxdu = (u >= -50.f && u <= 50.f) ? sg * fmaf(v, 1.f - sg, 1.f) : 0.f;
+    }
+    const float xc = fminf(fmaxf(x, -25.f), 25.f);
+    const float q = __expf(-xc), q2 = q * q;
+    const float rcp = __fdividef(1.f, (1.f + q) * (1.f + q2));
+    const float m = (1.f + q2) * rcp;
+    const float th = (1.f - q2) * (1.f + q) * rcp;
+    float sn, cs;
+    __sincosf(3.14159265358979f * th, &sn, &cs);
+    const bool open = act || u >= tau;           // with clamp + SiLU every gate is open (see the forward)
+    const float dm = fmaf(lr, cs, li * sn);
+    const float dph = (open ? m : 0.f) * fmaf(li, cs, -lr * sn);
+    const float dx = fmaf(dm * m, 1.f - m, dph * 3.14159265358979f * fmaf(-th, th, 1.f));
+    return dx * dxdu;
+}
+
 template <int T, int W, int KIND, bool VEC, bool DYN, bool FULL, bool EAR = false, int IO = IO_F32>
 __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, KIND, DYN> &sm,
                                           const int g, const int b, const int k)
 {
     static_assert(!(DYN && KIND == KIND_FUSED), "time-varying retention is not built for the fused path");
-    static_assert(!(EAR && (DYN || KIND == KIND_BWD)), "the Ear epilogue belongs to the static forward");
-    static_assert(IO == IO_F32 || (!EAR && !DYN && KIND != KIND_BWD), "bf16 storage is built for the static forward");
+    static_assert(!(EAR && (DYN || kind_is_bwd(KIND))), "the Ear epilogue belongs to the static forward");
+    static_assert(IO == IO_F32 || (!EAR && !DYN && !kind_is_bwd(KIND)), "bf16 storage is built for the static forward");
     constexpr bool IN16 = (IO & IO_IN_BF16) != 0, OUT16 = (IO & IO_OUT_BF16) != 0;
-    constexpr bool REV = (KIND == KIND_BWD);
+    static_assert(!(DYN && KIND == KIND_MIXBWD), "time-varying retention is not built for the fused path");
+    constexpr bool REV = kind_is_bwd(KIND);
+    constexpr bool MIX = (KIND == KIND_MIXBWD);
     constexpr int TILE = T * W;
     constexpr int M = kWindow;
     const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
@@ -270,7 +311,7 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
             __syncthreads();
         }
     }
-    const bool early = (KIND != KIND_BWD) && prm.early_loads != 0;
+    const bool early = !REV && prm.early_loads != 0;
     if (!early) grid_wait_previous();
     // Fused path: the hidden rows (floats) are staged in the upper part of the tile, behind
     // kHalo rows of history; phase 1 takes them into registers before the pushes overwrite them.
@@ -344,7 +385,33 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
             fetch_rows<VEC, T, GR>(xs, smem_addr(xs), reinterpret_cast<const char *>(prm.in) + e0 * 8, rowbytes, vA, vB,
                                    [&](int i) { return FULL || i < nvalid; });
     }
-    if constexpr (KIND == KIND_BWD) {
+    if constexpr (MIX) {
+        // hidden rows this tile's conv windows reach, in processing order: row R holds physical
+        // row t_hi - R (t_hi = the tile's last row in time); before t = 0 comes the carried
+        // history, before that zeros.  Each thread brings its own T rows, warp 0 the kHalo more.
+        const int Kh = prm.conv_k - 1;
+        const long long t_hi = L - 1 - (long long)k * TILE;
+        auto stage_h = [&](int R) {
+            const long long t = t_hi - R;
+            float *d = &sm.hrev[R][2 * lane];
+            const float *src = nullptr;
+            if (t >= 0) src = prm.hid + ((long long)b * L + t) * C + c0;
+            else if (t >= -Kh && prm.tail_in != nullptr) src = prm.tail_in + ((long long)b * Kh + (Kh + t)) * C + c0;
+            if (VEC) {
+                if (src != nullptr && vA) cp_async8<0>(smem_addr(d), src); else *reinterpret_cast<float2 *>(d) = make_float2(0.f, 0.f);
+            } else {
+                if (src != nullptr && vA) cp_async4(smem_addr(d), src); else d[0] = 0.f;
+                if (src != nullptr && vB) cp_async4(smem_addr(d + 1), src + 1); else d[1] = 0.f;
+            }
+        };
+#pragma unroll
+        for (int i = 0; i < T; ++i) stage_h(w * T + i);
+        if (w == 0) {
+#pragma unroll
+            for (int j = 0; j < kHalo; ++j) stage_h(TILE + j);
+        }
+    }
+    if constexpr (REV) {
         float4 *const qs = &sm.tile[1][w * T][lane];
         const bool have = prm.aux != nullptr;
         fetch_rows<VEC, T, 0>(qs, smem_addr(qs), reinterpret_cast<const char *>(prm.aux) + (e0 - C) * 8, rowbytes,
@@ -436,7 +503,7 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
         if (vB) { const float2 v = sp[1]; sinit.z = v.x; sinit.w = v.y; }
     }
 
-    if constexpr (KIND == KIND_BWD) {
+    if constexpr (REV) {
         cp_async_wait_all();
         // the step at t = 0 multiplies the call's initial state; lam_{L-1} = G_{L-1} + grad_state_out
         if (nvalid > 0 && t_first - (nvalid - 1) == 0 && prm.aux != nullptr && prm.state_in != nullptr) {
@@ -797,7 +864,45 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
         // the row processed before it), and the running sum of the logit gradient
         float2 gstep = make_float2(0.f, 0.f), sacc = make_float2(0.f, 0.f);
         if constexpr (DYN && REV) gstep = row_gamma(t_first + 1);
+        // MIXBWD: conv taps (right-aligned: tap j multiplies the hidden row 3 - j steps back), the
+        // rolling window of hidden rows, and the sums for the conv gradients
+        float mwA[4] = {}, mwB[4] = {}, mbA = 0.f, mbB = 0.f;
+        float2 hwin[4] = {};                             // h(t), h(t-1), h(t-2), h(t-3) of the current row
+        float caA[5] = {}, caB[5] = {};
+        const bool mact = prm.clamp_silu != 0;
+        if constexpr (MIX) {
+            const int Kc = prm.conv_k;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int kk = j - (4 - Kc);
+                mwA[j] = (kk >= 0 && vA) ? prm.conv_w[(long long)c0 * Kc + kk] : 0.f;
+                mwB[j] = (kk >= 0 && vB) ? prm.conv_w[(long long)(c0 + 1) * Kc + kk] : 0.f;
+            }
+            if (prm.conv_bias != nullptr) { if (vA) mbA = prm.conv_bias[c0]; if (vB) mbB = prm.conv_bias[c0 + 1]; }
+#pragma unroll
+            for (int r = 0; r < 3; ++r) hwin[r + 1] = *reinterpret_cast<const float2 *>(&sm.hrev[w * T + r][2 * lane]);
+        }
+        // one row of the MIXBWD form: lam -> du, kept in the row's (spent) input slot for the
+        // conv transpose that follows the loop
+        auto mix_row = [&](int i, float4 lam) {
+            hwin[0] = hwin[1]; hwin[1] = hwin[2]; hwin[2] = hwin[3];
+            hwin[3] = *reinterpret_cast<const float2 *>(&sm.hrev[w * T + i + 3][2 * lane]);
+            float uA = mbA, uB = mbB;
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if (j >= 4 - prm.conv_k) { uA = fmaf(mwA[j], hwin[3 - j].x, uA); uB = fmaf(mwB[j], hwin[3 - j].y, uB); }
+            const float duA = vA ? prelude_du(uA, lam.x, lam.y, mact, prm.gate_tau) : 0.f;
+            const float duB = vB ? prelude_du(uB, lam.z, lam.w, mact, prm.gate_tau) : 0.f;
+            xs[i * 32] = make_float4(duA, duB, 0.f, 0.f);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                caA[j] = fmaf(duA, hwin[3 - j].x, caA[j]);
+                caB[j] = fmaf(duB, hwin[3 - j].y, caB[j]);
+            }
+            caA[4] += duA; caB[4] += duB;
+        };
         auto step_row = [&](int i, bool clamped) {
+            if (MIX && !(FULL || i < nvalid)) xs[i * 32] = zero4();      // no such row: its du is 0
             if (FULL || i < nvalid) {
                 float2 gown = make_float2(0.f, 0.f);
                 if constexpr (DYN) {
@@ -807,8 +912,9 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
                 } else {
                     P = cfma2(a, P, xs[i * 32]);
                 }
-                store_row(i, clamped ? clamp4(P, cl) : P);
-                if constexpr (KIND == KIND_BWD) {
+                if constexpr (MIX) mix_row(i, clamped ? clamp4(P, cl) : P);
+                else store_row(i, clamped ? clamp4(P, cl) : P);
+                if constexpr (REV) {
                     // conj(lam) * P_{t-1}
                     const float4 q = sm.tile[1][w * T + i][lane];
                     if constexpr (DYN) {
@@ -881,6 +987,60 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
             if (vA) s[0] = make_float2(P.x, P.y);
             if (vB) s[1] = make_float2(P.z, P.w);
         }
+        if constexpr (MIX) {
+            // Transposed conv: grad_h(t) = sum_j w[j] du(t + 3 - j).  Row R of the tile (physical
+            // t_hi - R) needs du of rows R-3 .. R; the tile's first three rows would need the tile
+            // after it in time, so their du (and the du of its three earliest rows, for the tile
+            // before it) go to the edge area and a small kernel finishes those rows.
+            __syncthreads();
+            const float4 (*du)[32] = sm.tile[0];
+            float *const gh = reinterpret_cast<float *>(prm.out);
+#pragma unroll
+            for (int i = 0; i < T; ++i) {
+                const int R = w * T + i;
+                if ((FULL || i < nvalid) && R >= 3) {
+                    float dA = 0.f, dB = 0.f;
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const float2 d = *reinterpret_cast<const float2 *>(&du[R - 3 + j][lane]);
+                        dA = fmaf(mwA[j], d.x, dA); dB = fmaf(mwB[j], d.y, dB);
+                    }
+                    float *o = gh + (e0 - (long long)i * C);
+                    if (VEC) { if (vA) __stcs(reinterpret_cast<float2 *>(o), make_float2(dA, dB)); }
+                    else { if (vA) __stcs(o, dA); if (vB) __stcs(o + 1, dB); }
+                }
+            }
+            if (w == 0) {
+                const long long rem = L - (long long)k * TILE;
+                const int nrows = rem >= TILE ? TILE : (int)rem;           // rows this tile has
+                float *eg = prm.edge_du + (((long long)b * K + k) * 6) * C + c0;
+#pragma unroll
+                for (int r = 0; r < 3; ++r) {
+                    const float2 hi = r < nrows ? *reinterpret_cast<const float2 *>(&du[r][lane]) : make_float2(0.f, 0.f);
+                    const float2 lo = r < nrows ? *reinterpret_cast<const float2 *>(&du[nrows - 1 - r][lane]) : make_float2(0.f, 0.f);
+                    if (vA) { eg[(long long)r * C] = hi.x; eg[(long long)(3 + r) * C] = lo.x; }
+                    if (vB) { eg[(long long)r * C + 1] = hi.y; eg[(long long)(3 + r) * C + 1] = lo.y; }
+                }
+            }
+            if (prm.cpart != nullptr) {
+                // per-tile sums for the conv gradients, in a fixed order (the P tile is spent)
+                __syncthreads();
+                float *sp = reinterpret_cast<float *>(&sm.tile[1][0][0]);
+#pragma unroll
+                for (int j = 0; j < 5; ++j) { sp[(w * 32 + lane) * 10 + j] = caA[j]; sp[(w * 32 + lane) * 10 + 5 + j] = caB[j]; }
+                __syncthreads();
+                if (w == 0) {
+                    float *o = prm.cpart + (((long long)b * K + k) * C + c0) * 5;
+#pragma unroll
+                    for (int j = 0; j < 10; ++j) {
+                        float acc = 0.f;
+#pragma unroll
+                        for (int i = 0; i < W; ++i) acc += sp[(i * 32 + lane) * 10 + j];
+                        if (j < 5 ? vA : vB) o[j] = acc;
+                    }
+                }
+            }
+        }
     } else if (checkpoint && w == 0) {
         if constexpr (DYN) publish_pair_d(prm.pre + (chain * prm.KP + k / M) * 64, lane, zero4(), make_float2(0.f, 0.f), epoch, REC_POISON);
         else publish_pair(prm.pre + (chain * prm.KP + k / M) * 64, lane, zero4(), epoch, REC_POISON);
@@ -913,7 +1073,7 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
             }
         }
     }
-    if constexpr (KIND == KIND_BWD) {
+    if constexpr (REV) {
         if (prm.qpart != nullptr) {
             __syncthreads();
             sm.sE[w][lane] = qa;

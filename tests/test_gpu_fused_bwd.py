@@ -95,6 +95,15 @@ def test_mixing_bwd_shapes(B, L, C, Kc):
     compare(got, reference(d, 0.1, P_in=d["P_in"], gso_P=d["gso_P"], gso_tail=tail), L, Kc)
 
 
+@pytest.mark.parametrize("L", [15, 16, 17, 18, 19, 31, 32, 33, 34, 35, 63, 64, 65, 66, 67, 127, 128, 129, 130, 131, 192, 193])
+def test_mixing_bwd_rows_at_tile_seams(L):
+    """Lengths around multiples of the tile (16 rows up to L = 32, 64 beyond): the rows whose conv
+    transpose crosses a tile seam, a last tile of one to three rows, and the history gradient."""
+    d = make(2, L, 66, 4, seed=1200 + L)
+    got = run_mixing_bwd(d, 0.1, P_in=d["P_in"], gso_P=d["gso_P"], gso_tail=d["gso_tail"])
+    compare(got, reference(d, 0.1, P_in=d["P_in"], gso_P=d["gso_P"], gso_tail=d["gso_tail"]), L, 4)
+
+
 def test_mixing_bwd_clamp_silu_and_no_state():
     d = make(2, 400, 128, 4, seed=91, with_tail=False)
     d["h"] = (d["h"] * 20).astype(np.float32)
