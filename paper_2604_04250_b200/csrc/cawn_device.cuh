@@ -133,6 +133,26 @@ __device__ __forceinline__ float4 scale_step2(float4 a, float4 P, float2 g, floa
     const float4 t = cmul2(a, P);
     return make_float4(fmaf(g.x, t.x, x.x), fmaf(g.x, t.y, x.y), fmaf(g.y, t.z, x.z), fmaf(g.y, t.w, x.w));
 }
+// Single-instruction special functions in their flush-to-zero forms (no subnormal fix-up code
+// around them).  Callers keep arguments and results in the normal range: ex2 of |x| <= 40,
+// reciprocals of values in [1, 1e25], sines and cosines of |x| <= pi whose results only feed sums.
+__device__ __forceinline__ float ex2_ftz(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ float rcp_ftz(float x)
+{
+    float y;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ void sincos_ftz(float x, float &sn, float &cs)
+{
+    asm("sin.approx.ftz.f32 %0, %1;" : "=f"(sn) : "f"(x));
+    asm("cos.approx.ftz.f32 %0, %1;" : "=f"(cs) : "f"(x));
+}
 __device__ __forceinline__ float sigmoidf_fast(float s) { return __fdividef(1.f, 1.f + __expf(-s)); }
 
 // Records of the time-varying form: {re, im, factor product, tag} with a 32-bit tag
