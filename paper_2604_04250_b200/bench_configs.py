@@ -170,6 +170,18 @@ def _cfg3(args, cb, inputs, dev):
                args.steps, args.warmup)
     assert cb.cawn_poll_status(wb) == 0
     _report("cfg3_bwd", B * L, B * L * C * 24, ms, 2, {"note": "reads grad_y and saved P, writes grad_p; plus the finalize kernel"})
+    # the same backward with time-varying retention (logit and frequency-bias gradients)
+    dd = inputs.dynamic_retention_inputs(B, L, cfg.H, cfg.F, 7)
+    gl, fb = dev(dd["gamma_logit"]), dev(dd["freq_bias"])
+    prm_d = cb.make_params(B, L, cfg.H, cfg.F, gate_eps=cfg.gate_eps, flags=cb.CAWN_FLAG_RETENTION_DYNAMIC)
+    ggl, gfb = torch.empty((B, L, cfg.H), device="cuda"), torch.empty(cfg.F, device="cuda")
+    ms = _time(lambda i: cb.cawn_phase_accumulate_bwd_dynamic(prm_d, Ps[i % NS], cb.CAWN_SAVED_STATES, gl, fb, t, gys[i % NS],
+                                                              gps[i % NS], wb, grad_gamma_logit=ggl, grad_freq_bias=gfb,
+                                                              grad_theta=gt, grad_state_in=gsi),
+               args.steps, args.warmup)
+    assert cb.cawn_poll_status(wb) == 0
+    _report("cfg3_bwd_dynamic_retention", B * L, B * L * (C * 24 + cfg.H * 8), ms, 4,
+            {"note": "memset of the logit gradient, scan (atomic adds per row and head), two reductions"})
 
 
 def _cfg4(args, cb, inputs, dev, IND):

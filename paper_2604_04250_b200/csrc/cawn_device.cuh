@@ -153,7 +153,7 @@ __device__ __forceinline__ void sincos_ftz(float x, float &sn, float &cs)
     asm("sin.approx.ftz.f32 %0, %1;" : "=f"(sn) : "f"(x));
     asm("cos.approx.ftz.f32 %0, %1;" : "=f"(cs) : "f"(x));
 }
-__device__ __forceinline__ float sigmoidf_fast(float s) { return __fdividef(1.f, 1.f + __expf(-s)); }
+__device__ __forceinline__ float sigmoidf_fast(float s) { return rcp_ftz(1.f + ex2_ftz(s * -1.44269504088896f)); }
 
 // Records of the time-varying form: {re, im, factor product, tag} with a 32-bit tag
 // (epoch mod 2^30) * 4 + kind.

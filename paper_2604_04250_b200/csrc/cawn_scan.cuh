@@ -139,6 +139,7 @@ struct ScanSmem {
     float sCoef[64][6];
     float2 sD[DYN ? W : 1][DYN ? 32 : 1];             // DYN: factor products of the warps' steps
     float2 sRD[DYN ? kWindow + 1 : 1][DYN ? 32 : 1];  // DYN: factor products of the window's tiles
+    float2 sG[DYN ? TILE : 1][DYN ? 32 : 1];          // DYN: each row's own factor pair, kept from phase 1 for phase 3
     unsigned long long epoch;
     int err;
     int pad;
@@ -482,6 +483,7 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
         return gm;
     };
     float2 dprod = make_float2(1.f, 1.f);                // product of this thread's step factors
+    float2 gfirst = make_float2(0.f, 0.f);               // DYN backward: factor of the row before this thread's first
 
     // Window of carry records this tile needs (see the header comment), and a first,
     // non-blocking reading of the record this warp is responsible for: it is usually there
@@ -627,6 +629,19 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
         const bool want_mask = prm.mask != nullptr;
         uint32_t *const mrow0 = prm.mask + ((long long)b * L + s0) * prm.MW + g * 2;
         const bool second_word = g * 2 + 1 < prm.MW;
+        // DYN: the rows' retention logits, all requested up front so that their latencies overlap
+        float2 lg[DYN ? T : 1];
+        if constexpr (DYN) {
+#pragma unroll
+            for (int i = 0; i < T; ++i) {
+                lg[i] = make_float2(0.f, 0.f);
+                if (FULL || i < nvalid) {
+                    const float *gl = prm.gamma_logit + ((long long)b * L + s0 + i) * prm.H;
+                    if (vA) lg[i].x = gl[hA];
+                    if (vB) lg[i].y = gl[hB];
+                }
+            }
+        }
         auto pass = [&](auto exact_tag, auto mask_tag) -> float {
             constexpr bool EXACT = decltype(exact_tag)::value, MASK = decltype(mask_tag)::value;
             float nearest = INFINITY;
@@ -676,7 +691,9 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
                 }
                 if (FULL || i < nvalid) {
                     if constexpr (DYN) {
-                        const float2 gm = row_gamma(s0 + i);
+                        const float2 gm = make_float2(vA ? sigmoidf_fast(lg[i].x + fbA) : 0.f,
+                                                      vB ? sigmoidf_fast(lg[i].y + fbB) : 0.f);
+                        sm.sG[w * T + i][lane] = gm;
                         e = scale_step2(a, e, gm, v);
                         dprod.x *= gm.x; dprod.y *= gm.y;
                     } else {
@@ -700,13 +717,26 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
         if constexpr (DYN) {
             // moving from row t+1 to row t multiplies by gamma_{t+1} conj(R): the factor of the
             // row processed just before (row L does not exist: factor 0 on a zero carry)
+            // (the rows' logits are requested up front so that their latencies overlap)
+            float2 lgb[T];
+#pragma unroll
+            for (int i = 0; i < T; ++i) {
+                lgb[i] = make_float2(0.f, 0.f);
+                if (FULL || i < nvalid) {
+                    const float *gl = prm.gamma_logit + ((long long)b * L + (t_first - i)) * prm.H;
+                    if (vA) lgb[i].x = gl[hA];
+                    if (vB) lgb[i].y = gl[hB];
+                }
+            }
             float2 gm = row_gamma(t_first + 1);
+            gfirst = gm;
 #pragma unroll
             for (int i = 0; i < T; ++i) {
                 if (FULL || i < nvalid) {
                     e = scale_step2(a, e, gm, xs[i * 32]);
                     dprod.x *= gm.x; dprod.y *= gm.y;
-                    gm = row_gamma(t_first - i);
+                    gm = make_float2(vA ? sigmoidf_fast(lgb[i].x + fbA) : 0.f, vB ? sigmoidf_fast(lgb[i].y + fbB) : 0.f);
+                    sm.sG[w * T + i][lane] = gm;
                 }
             }
         } else {
@@ -863,7 +893,7 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
         // DYN: factor of the step into row i (forward: the row's own; backward: the factor of
         // the row processed before it), and the running sum of the logit gradient
         float2 gstep = make_float2(0.f, 0.f), sacc = make_float2(0.f, 0.f);
-        if constexpr (DYN && REV) gstep = row_gamma(t_first + 1);
+        if constexpr (DYN && REV) gstep = gfirst;
         // MIXBWD: conv taps (right-aligned: tap j multiplies the hidden row 3 - j steps back), the
         // rolling window of hidden rows, and the sums for the conv gradients
         float mwA[4] = {}, mwB[4] = {}, mbA = 0.f, mbB = 0.f;
@@ -906,9 +936,9 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
             if (FULL || i < nvalid) {
                 float2 gown = make_float2(0.f, 0.f);
                 if constexpr (DYN) {
-                    if (!REV) gstep = row_gamma(s0 + i);
+                    if (!REV) gstep = sm.sG[w * T + i][lane];
                     P = scale_step2(a, P, gstep, xs[i * 32]);
-                    if (REV) { gown = row_gamma(t_first - i); gstep = gown; }
+                    if (REV) { gown = sm.sG[w * T + i][lane]; gstep = gown; }
                 } else {
                     P = cfma2(a, P, xs[i * 32]);
                 }
