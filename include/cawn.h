@@ -55,8 +55,14 @@ typedef enum cawn_status {
     CAWN_ERR_CUDA                 = -6,  /* a CUDA runtime call failed (launch, copy)            */
     CAWN_ERR_STATIC_TOO_LARGE     = -7,  /* cawn_phase_accumulate_fwd_static: the call needs more
                                             scratch than the library's built-in array holds      */
-    CAWN_ERR_CARRY_TIMEOUT        = 1    /* device: an inter-tile carry wait hit its bound;
+    CAWN_ERR_CARRY_TIMEOUT        = 1,   /* device: an inter-tile carry wait hit its bound;
                                             outputs of that call are incomplete                  */
+    CAWN_STATUS_NONFINITE         = 2    /* device: an Inf or NaN was accumulated (an Inf input, a
+                                            non-finite carried state, an overflow); outputs are
+                                            complete but contain such values.  NaN pushes alone do
+                                            not raise it: they fail the gate's comparison and are
+                                            dropped.  The two device conditions are bits: a poll may
+                                            return 3 when both occurred.                          */
 } cawn_status;
 
 enum {
@@ -288,8 +294,22 @@ CAWN_API int cawn_state_carry(const cawn_params *params,
                               void *state_out, void *cuda_stream);
 
 /* Synchronise `cuda_stream` and return the device-side status recorded in the workspace by
- * the calls so far (CAWN_OK or a positive cawn_status); the record is then cleared.            */
+ * the calls so far (CAWN_OK, or the positive conditions CAWN_ERR_CARRY_TIMEOUT and
+ * CAWN_STATUS_NONFINITE or-ed together); the record is then cleared.  This is the hook for the
+ * paper's stability protocol (Section "Training Stability in the Complex Domain": skip the step
+ * on NaN/Inf), without a pass over the outputs.                                                    */
 CAWN_API int cawn_poll_status(void *workspace, void *cuda_stream);
+
+/* Test hook for the bounded waits (no counterpart in the paper).  After this call, in every
+ * kernel that uses `workspace`, tile number `withhold_tile` (0-based along time, in the kernel's
+ * own tile size: 128 steps in the forward, 64 in the backward, 16 for calls of at most 32 steps)
+ * of every (batch, channel group) keeps its summary to itself, and every carry wait gives up
+ * after `poll_bound` polls (1..65535; 0 keeps the normal bound).  Tiles that depend on the silent
+ * one then run into the bound, record CAWN_ERR_CARRY_TIMEOUT, skip their outputs and pass the
+ * failure on; the kernel ends, nothing hangs or traps, and the workspace stays usable.
+ * withhold_tile < 0 and poll_bound = 0 switch the hook off.  Stream-ordered.                   */
+CAWN_API int cawn_workspace_set_wait_hook(void *workspace, int withhold_tile, unsigned poll_bound,
+                                          void *cuda_stream);
 
 /*
  * Host-buffer convenience for the Cartesian forward: copies pushes, gamma, theta (and

@@ -23,6 +23,7 @@ CAWN_ERR_CUDA = -6
 CAWN_ERR_STATIC_TOO_LARGE = -7
 CAWN_STATIC_SCRATCH_BYTES = 4 << 20
 CAWN_ERR_CARRY_TIMEOUT = 1
+CAWN_STATUS_NONFINITE = 2
 
 CAWN_FLAG_PRELUDE_CLAMP_SILU = 1
 CAWN_FLAG_RETENTION_DYNAMIC = 2
@@ -38,6 +39,7 @@ EXPORTS = (
     "cawn_phase_accumulate_fwd", "cawn_phase_accumulate_bwd", "cawn_state_carry",
     "cawn_poll_status", "cawn_phase_accumulate_fwd_host", "cawn_phase_accumulate_fwd_static",
     "cawn_phase_accumulate_bwd_dynamic", "cawn_mixing_bwd", "cawn_phase_accumulate_fwd_ear",
+    "cawn_workspace_set_wait_hook",
 )
 
 
@@ -88,6 +90,7 @@ def lib():
         L.cawn_phase_accumulate_fwd_ear.argtypes = [pp, vp, fp, fp, fp, fp, vp, fp, fp, ctypes.c_int, fp, vp, vp, vp, sz, vp]
         L.cawn_state_carry.argtypes = [pp, vp, vp, ctypes.c_int64, fp, fp, vp, vp]
         L.cawn_poll_status.argtypes = [vp, vp]
+        L.cawn_workspace_set_wait_hook.argtypes = [vp, ctypes.c_int, ctypes.c_uint, vp]
         L.cawn_phase_accumulate_fwd_host.argtypes = [pp, vp, fp, fp, vp, vp, vp, vp, vp, sz, vp]
         L.cawn_phase_accumulate_fwd_static.argtypes = [pp, vp, fp, fp, vp, vp, vp, vp, vp, vp]
         for name in EXPORTS:
@@ -182,6 +185,11 @@ def cawn_state_carry(params, state_prev, state_local, n_steps, gamma, theta, sta
     _check(lib().cawn_state_carry(ctypes.byref(params), _dp(state_prev), _dp(state_local),
                                   int(n_steps), _dp(gamma), _dp(theta), _dp(state_out),
                                   _stream(stream)), "cawn_state_carry")
+
+
+def cawn_workspace_set_wait_hook(workspace, withhold_tile, poll_bound, stream=None):
+    _check(lib().cawn_workspace_set_wait_hook(_dp(workspace), int(withhold_tile), int(poll_bound), _stream(stream)),
+           "cawn_workspace_set_wait_hook")
 
 
 def cawn_poll_status(workspace, stream=None):

@@ -221,6 +221,8 @@ const char *cawn_status_string(int status)
     case CAWN_ERR_CUDA: return "CUDA runtime error";
     case CAWN_ERR_STATIC_TOO_LARGE: return "call needs more scratch than the built-in array holds";
     case CAWN_ERR_CARRY_TIMEOUT: return "device: inter-tile carry wait ran out";
+    case CAWN_STATUS_NONFINITE: return "device: non-finite values seen";
+    case CAWN_ERR_CARRY_TIMEOUT | CAWN_STATUS_NONFINITE: return "device: inter-tile carry wait ran out; non-finite values seen";
     default: return "unknown status";
     }
 }
@@ -666,6 +668,16 @@ int cawn_poll_status(void *workspace, void *cuda_stream)
         if (cudaStreamSynchronize(st) != cudaSuccess) return CAWN_ERR_CUDA;
     }
     return (int)status;
+}
+
+int cawn_workspace_set_wait_hook(void *workspace, int withhold_tile, unsigned poll_bound, void *cuda_stream)
+{
+    if (workspace == nullptr) return CAWN_ERR_NULL_POINTER;
+    if (withhold_tile >= 65535 || poll_bound > 65535u) return CAWN_ERR_INVALID_ARG;
+    const unsigned word = (poll_bound << 16) | (withhold_tile < 0 ? 0u : (unsigned)withhold_tile + 1u);
+    WsHeader *ws = reinterpret_cast<WsHeader *>(workspace);
+    cawn_set_word_kernel<<<1, 1, 0, (cudaStream_t)cuda_stream>>>(&ws->hook, word);
+    return cudaGetLastError() == cudaSuccess ? CAWN_OK : CAWN_ERR_CUDA;
 }
 
 int cawn_phase_accumulate_fwd_host(const cawn_params *params, const void *p_host,

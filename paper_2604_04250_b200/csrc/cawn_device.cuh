@@ -13,16 +13,29 @@ namespace cawn {
 //          launches (and a launch replayed from a CUDA graph still sees a fresh epoch).
 // done   : CTAs of the current launch that have read the epoch.  The last one to arrive
 //          resets the count and opens the next epoch; by then nobody reads `epoch` any more.
-// status : sticky device-side error (cawn_status > 0), cleared by cawn_poll_status.
+// status : sticky device-side conditions (bits: STATUS_CARRY_TIMEOUT, STATUS_NONFINITE), cleared by
+//          cawn_poll_status.
+// hook   : test hook for the bounded waits, 0 = off: low 16 bits = 1 + index of the tile (of every
+//          chain) that does not publish its aggregate, high 16 bits = poll bound to use instead
+//          of the normal one.  Only cawn_workspace_set_wait_hook writes it.
 struct __align__(16) WsHeader {
     unsigned long long epoch;
+    unsigned int hook;           // next to the epoch: a CTA reads both with one 16-byte load
     unsigned int done;
     unsigned int status;
-    unsigned int reserved[60];
+    unsigned int reserved[59];
 };
 static_assert(sizeof(WsHeader) == 256, "workspace header is 256 bytes");
 
 enum : unsigned { REC_AGGREGATE = 1u, REC_PREFIX = 2u, REC_POISON = 3u };
+enum : unsigned { STATUS_CARRY_TIMEOUT = 1u, STATUS_NONFINITE = 2u };
+
+// true unless all four components are finite (their sum is then finite too, short of overflow,
+// which is reported just the same)
+__device__ __forceinline__ bool nonfinite4(float4 v)
+{
+    return !(fabsf((v.x + v.y) + (v.z + v.w)) < INFINITY);
+}
 
 // ---------------------------------------------------------------------------------------
 // Every lane works on two adjacent channels at once; a float4 holds (re0, im0, re1, im1).
@@ -70,11 +83,13 @@ __device__ __forceinline__ uint4 ld_record(const uint4 *p)
                  : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
     return v;
 }
-__device__ __forceinline__ unsigned long long ld_volatile_u64(const unsigned long long *p)
+// epoch and hook of a workspace header in one access
+__device__ __forceinline__ void ld_epoch_hook(const void *hdr, unsigned long long &epoch, unsigned &hook)
 {
-    unsigned long long v;
-    asm volatile("ld.volatile.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
-    return v;
+    unsigned x, y, z, w;
+    asm volatile("ld.volatile.global.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(x), "=r"(y), "=r"(z), "=r"(w) : "l"(hdr) : "memory");
+    epoch = ((unsigned long long)y << 32) | x;
+    hook = z;
 }
 __device__ __forceinline__ void st_volatile_u64(unsigned long long *p, unsigned long long v)
 {

@@ -142,7 +142,7 @@ struct ScanSmem {
     float2 sG[DYN ? TILE : 1][DYN ? 32 : 1];          // DYN: each row's own factor pair, kept from phase 1 for phase 3
     unsigned long long epoch;
     int err;
-    int pad;
+    unsigned hook;                                     // copy of the workspace's wait hook
 };
 
 __device__ __forceinline__ uint32_t smem_addr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -446,9 +446,11 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
     unsigned long long epoch0 = 0;
     unsigned arrived = 0;
     if (tid == 0) {
-        epoch0 = ld_volatile_u64(&prm.ws->epoch);
+        unsigned hook0;
+        ld_epoch_hook(prm.ws, epoch0, hook0);
         sm.epoch = epoch0;
         sm.err = 0;
+        sm.hook = hook0;
         // counted only once the epoch has been read (the increment depends on its value)
         arrived = atomicAdd(&prm.ws->done, 1u + (unsigned)(epoch0 >> 63));
     }
@@ -755,7 +757,10 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
     __syncthreads();                                                           // barrier 2
 
     // ---- 2. publish the aggregate, fetch the carry window ----------------------------------
-    if (w == 0 && k + 1 < K) {
+    const unsigned hook = sm.hook;
+    const unsigned poll_limit = (hook >> 16) != 0u ? (hook >> 16) : prm.poll_limit;
+    const bool withheld = (hook & 0xffffu) == (unsigned)k + 1u;      // test hook: this tile stays silent
+    if (w == 0 && k + 1 < K && !withheld) {
         float4 E = sm.sE[0][lane];
         if constexpr (DYN) {
             float2 D = sm.sD[0][lane];
@@ -781,13 +786,13 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
         float2 rd = make_float2(0.f, 0.f);
         if (slot < nrec) {
             const uint4 *rec = prm.agg + (chain * K + (k - 1 - slot)) * 64;
-            if constexpr (DYN) ok = poll_pair_d(rec, lane, epoch, prm.poll_limit, mine ? er0 : none, mine ? er1 : none, r, rd);
-            else ok = poll_pair(rec, lane, epoch, prm.poll_limit, mine ? er0 : none, mine ? er1 : none, r);
+            if constexpr (DYN) ok = poll_pair_d(rec, lane, epoch, poll_limit, mine ? er0 : none, mine ? er1 : none, r, rd);
+            else ok = poll_pair(rec, lane, epoch, poll_limit, mine ? er0 : none, mine ? er1 : none, r);
         } else if (slot == M) {
             if (cpt > 0) {
                 const uint4 *rec = prm.pre + (chain * prm.KP + cpt / M) * 64;
-                if constexpr (DYN) ok = poll_pair_d(rec, lane, epoch, prm.poll_limit, mine ? er0 : none, mine ? er1 : none, r, rd);
-                else ok = poll_pair(rec, lane, epoch, prm.poll_limit, mine ? er0 : none, mine ? er1 : none, r);
+                if constexpr (DYN) ok = poll_pair_d(rec, lane, epoch, poll_limit, mine ? er0 : none, mine ? er1 : none, r, rd);
+                else ok = poll_pair(rec, lane, epoch, poll_limit, mine ? er0 : none, mine ? er1 : none, r);
             } else {
                 r = sinit;
             }
@@ -796,7 +801,7 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
         if constexpr (DYN) sm.sRD[slot][lane] = rd;
         if (!ok) {
             sm.err = 1;
-            atomicMax(&prm.ws->status, 1u);              // CAWN_ERR_CARRY_TIMEOUT
+            atomicOr(&prm.ws->status, STATUS_CARRY_TIMEOUT);
         }
     }
     __syncthreads();                                                           // barrier 3
@@ -1007,6 +1012,10 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
             for (int i = 0; i < T; ++i) step_row(i, false);
         }
         sacc_out = sacc;
+        // An Inf or NaN that entered anywhere (an input, the carried state, an overflow) is still
+        // in the chain's last state: the recurrence never makes it finite again.  (A NaN push
+        // itself fails the gate's comparison and is dropped like any closed gate.)
+        if (nvalid > 0 && s0 + nvalid == L && nonfinite4(P)) atomicOr(&prm.ws->status, STATUS_NONFINITE);
         // the thread that owns the last step writes the carried state (never clamped)
         if (prm.state_out != nullptr && nvalid > 0 && s0 + nvalid == L) {
             if (REV) {                                   // grad_state_in = conj(a_0) lam_0

@@ -157,4 +157,7 @@ __global__ void cawn_conv_grad_finalize_kernel(const float *part, int nparts, in
     }
 }
 
+// One 32-bit word, stream-ordered (the wait hook of a workspace header).
+__global__ void cawn_set_word_kernel(unsigned *word, unsigned value) { *word = value; }
+
 }  // namespace cawn
