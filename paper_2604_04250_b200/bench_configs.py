@@ -145,6 +145,16 @@ def _decode(args, cb, inputs, dev):
     assert cb.cawn_poll_status(ws) == 0
     _report("decode_fused_B1_L1", n, n * C * 12, ms, n, {"us_per_token": ms * 1e3 / n,
             "note": "one launch per token; latency-bound, bandwidth figures are not meaningful"})
+    # the same n steps recorded once into a CUDA graph and replayed
+    side = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        gen(0)
+    ms = _time(lambda i: graph.replay(), max(args.steps // 10, 3), 2)
+    assert cb.cawn_poll_status(ws) == 0
+    _report("decode_fused_B1_L1_cuda_graph", n, n * C * 12, ms, n, {"us_per_token": ms * 1e3 / n,
+            "note": "256 decode steps replayed from one CUDA graph"})
 
 
 def _cfg3(args, cb, inputs, dev):
