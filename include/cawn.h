@@ -317,6 +317,13 @@ CAWN_API int cawn_workspace_set_wait_hook(void *workspace, int withhold_tile, un
  * (and state_out, gate_mask) back to HOST memory, all on `cuda_stream`, and returns without
  * synchronising.  `device_scratch` (device, >= cawn_workspace_bytes(CAWN_OP_FWD_HOST), zeroed
  * once with cawn_workspace_init) holds staging and workspace.  Static retention, conv_k == 0.
+ * Calls of 8 MB and more are cut into up to 8 slices (batch rows, or for B = 1 stretches of time
+ * with the state carried: the paper's chunked prefill) that go through two library-owned copy
+ * streams, so that slice i is copied out while slice i+1 is copied in; both streams wait for
+ * what precedes the call on `cuda_stream` and `cuda_stream` waits for both before anything
+ * after it.  The host buffers should be page-locked for the copies to overlap.  The copy streams
+ * and their events are created on the first such call per device (the only resources the
+ * library ever creates) and calls that use them are serialised by a lock.
  */
 CAWN_API int cawn_phase_accumulate_fwd_host(const cawn_params *params,
                                             const void *p_host,

@@ -6,6 +6,8 @@
 #include <math.h>
 #include <string.h>
 
+#include <mutex>
+
 namespace {
 
 using namespace cawn;
@@ -680,6 +682,39 @@ int cawn_workspace_set_wait_hook(void *workspace, int withhold_tile, unsigned po
     return cudaGetLastError() == cudaSuccess ? CAWN_OK : CAWN_ERR_CUDA;
 }
 
+// Copy pipes of the host-staged forward: one stream for host-to-device copies and kernels, one
+// for device-to-host copies, so that the two directions of the bus work at the same time.  One
+// set per device, created on first use and kept; calls that use them are serialised.
+constexpr int kHostSlices = 8;
+struct CopyPipes {
+    cudaStream_t in, out;
+    cudaEvent_t fork, in_done, out_done, slice[kHostSlices];
+    bool ready;
+};
+static std::mutex g_pipes_mutex;
+static CopyPipes g_pipes[64];
+
+static cudaError_t get_pipes(CopyPipes **out)
+{
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    CopyPipes &p = g_pipes[dev];
+    if (!p.ready) {
+        if ((e = cudaStreamCreateWithFlags(&p.in, cudaStreamNonBlocking)) != cudaSuccess) return e;
+        if ((e = cudaStreamCreateWithFlags(&p.out, cudaStreamNonBlocking)) != cudaSuccess) return e;
+        cudaEvent_t *ev[3] = {&p.fork, &p.in_done, &p.out_done};
+        for (int i = 0; i < 3; ++i)
+            if ((e = cudaEventCreateWithFlags(ev[i], cudaEventDisableTiming)) != cudaSuccess) return e;
+        for (int i = 0; i < kHostSlices; ++i)
+            if ((e = cudaEventCreateWithFlags(&p.slice[i], cudaEventDisableTiming)) != cudaSuccess) return e;
+        p.ready = true;
+    }
+    *out = &p;
+    return cudaSuccess;
+}
+
 int cawn_phase_accumulate_fwd_host(const cawn_params *params, const void *p_host,
                                    const float *gamma_host, const float *theta_host,
                                    const void *state_in_host, void *y_host, void *state_out_host,
@@ -698,34 +733,102 @@ int cawn_phase_accumulate_fwd_host(const cawn_params *params, const void *p_host
     if (device_scratch_bytes < h.total) return CAWN_ERR_WORKSPACE_TOO_SMALL;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     char *d = reinterpret_cast<char *>(device_scratch);
-    const size_t C = (size_t)params->H * params->F;
+    const size_t C = (size_t)params->H * params->F, MW = (C + 31) / 32;
     const size_t n = (size_t)params->B * (size_t)params->L * C;
     const size_t state_bytes = (size_t)params->B * C * sizeof(float2);
-    const size_t mask_bytes = (size_t)params->B * (size_t)params->L * ((C + 31) / 32) * sizeof(uint32_t);
+
+    // Slices that can be copied in, scanned and copied out one after another: batch rows when
+    // there are several (independent), else stretches of time with the state carried from one
+    // to the next (chunked prefill inside the call).  Small calls are one slice.
+    const bool by_batch = params->B >= 2;
+    int S = 1;
+    if (by_batch) {
+        S = params->B < kHostSlices ? params->B : kHostSlices;
+    } else {
+        const size_t want = n * sizeof(float2) / ((size_t)4 << 20);
+        S = want < 1 ? 1 : (want > (size_t)kHostSlices ? kHostSlices : (int)want);
+    }
+    if (n * sizeof(float2) < ((size_t)8 << 20)) S = 1;
+
+    CopyPipes *pp = nullptr;
+    std::unique_lock<std::mutex> lock(g_pipes_mutex, std::defer_lock);
+    cudaStream_t s_in = st, s_out = st;
     bool ok = true;
-    ok &= cudaMemcpyAsync(d + h.off_gamma, gamma_host, C * sizeof(float), cudaMemcpyHostToDevice, st) == cudaSuccess;
-    ok &= cudaMemcpyAsync(d + h.off_theta, theta_host, C * sizeof(float), cudaMemcpyHostToDevice, st) == cudaSuccess;
+    if (S > 1) {
+        lock.lock();
+        if (get_pipes(&pp) != cudaSuccess) return CAWN_ERR_CUDA;
+        s_in = pp->in; s_out = pp->out;
+        ok &= cudaEventRecord(pp->fork, st) == cudaSuccess;
+        ok &= cudaStreamWaitEvent(s_in, pp->fork, 0) == cudaSuccess;
+        ok &= cudaStreamWaitEvent(s_out, pp->fork, 0) == cudaSuccess;
+    }
+    ok &= cudaMemcpyAsync(d + h.off_gamma, gamma_host, C * sizeof(float), cudaMemcpyHostToDevice, s_in) == cudaSuccess;
+    ok &= cudaMemcpyAsync(d + h.off_theta, theta_host, C * sizeof(float), cudaMemcpyHostToDevice, s_in) == cudaSuccess;
     if (state_in_host)
-        ok &= cudaMemcpyAsync(d + h.off_state, state_in_host, state_bytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
-    if (n)
-        ok &= cudaMemcpyAsync(d + h.off_x, p_host, n * sizeof(float2), cudaMemcpyHostToDevice, st) == cudaSuccess;
+        ok &= cudaMemcpyAsync(d + h.off_state, state_in_host, state_bytes, cudaMemcpyHostToDevice, s_in) == cudaSuccess;
     if (!ok) return CAWN_ERR_CUDA;
-    rc = cawn_phase_accumulate_fwd(params, d + h.off_x,
-                                   reinterpret_cast<const float *>(d + h.off_gamma),
-                                   reinterpret_cast<const float *>(d + h.off_theta),
-                                   nullptr, nullptr, nullptr, nullptr,
-                                   state_in_host ? d + h.off_state : nullptr,
-                                   d + h.off_x,                               /* in place */
-                                   state_out_host ? d + h.off_state : nullptr,
-                                   gate_mask_host ? reinterpret_cast<uint32_t *>(d + h.off_mask) : nullptr,
-                                   d + h.off_ws, h.total - h.off_ws, st);
-    if (rc != CAWN_OK) return rc;
-    if (n)
-        ok &= cudaMemcpyAsync(y_host, d + h.off_x, n * sizeof(float2), cudaMemcpyDeviceToHost, st) == cudaSuccess;
+
+    const int64_t rows_total = by_batch ? params->B : params->L;       // what the slices divide
+    int64_t per = (rows_total + S - 1) / S;
+    if (!by_batch && S > 1) per = (per + 127) / 128 * 128;              // whole tiles per stretch of time
+    int64_t r0 = 0;
+    for (int i = 0; i < S && (r0 < rows_total || i == 0); ++i) {
+        const int64_t r1 = (r0 + per < rows_total) ? r0 + per : rows_total;
+        cawn_params q = *params;
+        size_t x_off, m_off, s_off = 0;
+        bool have_state = state_in_host != nullptr;
+        if (by_batch) {
+            q.B = (int32_t)(r1 - r0);
+            x_off = (size_t)r0 * (size_t)params->L * C;
+            m_off = (size_t)r0 * (size_t)params->L * MW;
+            s_off = (size_t)r0 * C;
+        } else {
+            q.L = r1 - r0;
+            x_off = (size_t)r0 * C;
+            m_off = (size_t)r0 * MW;
+            have_state = have_state || i > 0;                           // later stretches continue the first
+        }
+        const size_t nx = (size_t)q.B * (size_t)q.L * C;
+        char *x_dev = d + h.off_x + x_off * sizeof(float2);
+        char *state_dev = d + h.off_state + s_off * sizeof(float2);
+        uint32_t *mask_dev = reinterpret_cast<uint32_t *>(d + h.off_mask) + m_off;
+        const bool need_state_out = state_out_host != nullptr || (!by_batch && S > 1);
+        if (nx)
+            ok &= cudaMemcpyAsync(x_dev, reinterpret_cast<const char *>(p_host) + x_off * sizeof(float2), nx * sizeof(float2),
+                                  cudaMemcpyHostToDevice, s_in) == cudaSuccess;
+        if (!ok) return CAWN_ERR_CUDA;
+        rc = cawn_phase_accumulate_fwd(&q, x_dev,
+                                       reinterpret_cast<const float *>(d + h.off_gamma),
+                                       reinterpret_cast<const float *>(d + h.off_theta),
+                                       nullptr, nullptr, nullptr, nullptr,
+                                       have_state ? state_dev : nullptr,
+                                       x_dev,                                  /* in place */
+                                       need_state_out ? state_dev : nullptr,
+                                       gate_mask_host ? mask_dev : nullptr,
+                                       d + h.off_ws, h.total - h.off_ws, s_in);
+        if (rc != CAWN_OK) return rc;
+        if (S > 1) {
+            ok &= cudaEventRecord(pp->slice[i], s_in) == cudaSuccess;
+            ok &= cudaStreamWaitEvent(s_out, pp->slice[i], 0) == cudaSuccess;
+        }
+        if (nx)
+            ok &= cudaMemcpyAsync(reinterpret_cast<char *>(y_host) + x_off * sizeof(float2), x_dev, nx * sizeof(float2),
+                                  cudaMemcpyDeviceToHost, s_out) == cudaSuccess;
+        if (gate_mask_host && nx)
+            ok &= cudaMemcpyAsync(gate_mask_host + m_off, mask_dev, (size_t)q.B * (size_t)q.L * MW * sizeof(uint32_t),
+                                  cudaMemcpyDeviceToHost, s_out) == cudaSuccess;
+        if (!ok) return CAWN_ERR_CUDA;
+        r0 = r1;
+    }
+    // the state leaves after the last slice (s_out has waited for it)
     if (state_out_host)
-        ok &= cudaMemcpyAsync(state_out_host, d + h.off_state, state_bytes, cudaMemcpyDeviceToHost, st) == cudaSuccess;
-    if (gate_mask_host && mask_bytes)
-        ok &= cudaMemcpyAsync(gate_mask_host, d + h.off_mask, mask_bytes, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+        ok &= cudaMemcpyAsync(state_out_host, d + h.off_state, state_bytes, cudaMemcpyDeviceToHost, s_out) == cudaSuccess;
+    if (S > 1) {                                     // join both pipes back into the caller's stream
+        ok &= cudaEventRecord(pp->in_done, s_in) == cudaSuccess;
+        ok &= cudaEventRecord(pp->out_done, s_out) == cudaSuccess;
+        ok &= cudaStreamWaitEvent(st, pp->in_done, 0) == cudaSuccess;
+        ok &= cudaStreamWaitEvent(st, pp->out_done, 0) == cudaSuccess;
+    }
     return ok ? CAWN_OK : CAWN_ERR_CUDA;
 }
 

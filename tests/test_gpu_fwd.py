@@ -167,6 +167,31 @@ def test_host_buffer_entry_point():
     assert np.array_equal(unpack_mask(m.numpy().view(np.uint32), C), m_ref)
 
 
+@pytest.mark.parametrize("B,L,C", [(4, 4096, 128), (11, 2048, 64), (1, 20000, 128), (1, 9000, 192)])
+def test_host_buffer_entry_point_sliced(B, L, C):
+    """Calls of 8 MB and more go through the two copy streams in slices: batch rows for B >= 2,
+    stretches of time with the state carried for B = 1.  Two calls in a row reuse the pipes."""
+    import torch
+    from paper_2604_04250_b200 import binding as cb
+    d = inputs.scan_inputs(B, L, C, seed=150 + B, with_state=True)
+    prm = cb.make_params(B, L, 1, C, gate_eps=0.1)
+    scratch = cb.new_workspace(prm, cb.CAWN_OP_FWD_HOST)
+    pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+    p, g, t, si = pin(d["p"]), pin(d["gamma"]), pin(d["theta"]), pin(d["state_in"])
+    y_ref, so_ref, m_ref = oracle.forward(d["p"], d["gamma"], d["theta"], 0.1,
+                                          state_in=d["state_in"].astype(np.complex128))
+    for _ in range(2):
+        y = torch.full((B, L, C), float("nan"), dtype=torch.complex64).pin_memory()
+        so = torch.full((B, C), float("nan"), dtype=torch.complex64).pin_memory()
+        m = torch.zeros((B, L, C // 32), dtype=torch.int32).pin_memory()
+        cb.cawn_phase_accumulate_fwd_host(prm, p, g, t, y, scratch, state_in_host=si,
+                                          state_out_host=so, gate_mask_host=m)
+        torch.cuda.current_stream().synchronize()        # the caller's stream alone: the call joined its pipes into it
+        assert floored_rel_err(y.numpy(), y_ref, axes=(0, 1)) < TOL
+        assert floored_rel_err(so.numpy(), so_ref) < TOL
+        assert np.array_equal(unpack_mask(m.numpy().view(np.uint32), C), m_ref)
+
+
 def test_repeatable_bitwise():
     from gpu_util import run_fwd
     d = inputs.scan_inputs(4, 2048, 256, seed=16)
