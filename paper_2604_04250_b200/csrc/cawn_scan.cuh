@@ -262,7 +262,9 @@ __device__ __forceinline__ float prelude_du(float u, float lr, float li, bool ac
     return dx * dxdu;
 }
 
-template <int T, int W, int KIND, bool VEC, bool DYN, bool FULL, bool EAR = false, int IO = IO_F32>
+// MASKED = false compiles the gate-mask output out (the caller then never passes a mask), which
+// keeps its registers out of the plain forward.
+template <int T, int W, int KIND, bool VEC, bool DYN, bool FULL, bool EAR = false, int IO = IO_F32, bool MASKED = true>
 __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, KIND, DYN> &sm,
                                           const int g, const int b, const int k)
 {
@@ -558,7 +560,8 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
         const bool act = prm.clamp_silu != 0;
         const float tau = prm.gate_tau;
         const bool want_mask = prm.mask != nullptr;
-        uint32_t *mrow = prm.mask + ((long long)b * L + s0) * prm.MW + g * 2;
+        uint32_t *const mrow0 = prm.mask + ((long long)b * L + s0) * prm.MW + g * 2;
+        unsigned mkeep = 0u;                              // lane r: word 0 of row r; lane 16 + r: word 1
         const bool second_word = g * 2 + 1 < prm.MW;
         // All of it runs two channels wide on packed fp32 pairs (fma.rn.f32x2 and friends): a
         // lane's hidden values already come as (channel, channel+1) pairs, and the pushes are
@@ -606,11 +609,14 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
                 const unsigned bits = ((oA ? 1u : 0u) | (oB ? 2u : 0u)) << (2 * (lane & 15));
                 const unsigned w0 = __reduce_or_sync(0xffffffffu, lane < 16 ? bits : 0u);
                 const unsigned w1 = __reduce_or_sync(0xffffffffu, lane < 16 ? 0u : bits);
-                if (FULL || i < nvalid) {
-                    if (lane == 0) mrow[0] = w0;
-                    if (lane == 16 && second_word) mrow[1] = w1;
+                // rows are parked in lanes and stored sixteen at a time
+                if (lane == (i & 15)) mkeep = w0;
+                if (lane == 16 + (i & 15)) mkeep = w1;
+                if ((i & 15) == 15 || i == T - 1) {
+                    const int r = i - (i & 15) + (lane & 15);
+                    if ((lane & 15) <= (i & 15) && (FULL || r < nvalid) && (lane < 16 || second_word))
+                        mrow0[(long long)r * prm.MW + (lane >> 4)] = mkeep;
                 }
-                mrow += prm.MW;
             }
             if (FULL || i < nvalid) {
                 const float2 nr = __ffma2_rn(ar2, er2, __ffma2_rn(nai2, ei2, zr));
@@ -628,7 +634,7 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
         // the warp saw one inside the band, the warp redoes its rows with the double comparison
         // (shared memory still holds the original of every element the first pass kept).
         const float mid = prm.gate_mid, hw = prm.gate_hw, keep = prm.gate_keep;
-        const bool want_mask = prm.mask != nullptr;
+        const bool want_mask = MASKED && prm.mask != nullptr;
         uint32_t *const mrow0 = prm.mask + ((long long)b * L + s0) * prm.MW + g * 2;
         const bool second_word = g * 2 + 1 < prm.MW;
         // DYN: the rows' retention logits, all requested up front so that their latencies overlap
@@ -647,7 +653,7 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
         auto pass = [&](auto exact_tag, auto mask_tag) -> float {
             constexpr bool EXACT = decltype(exact_tag)::value, MASK = decltype(mask_tag)::value;
             float nearest = INFINITY;
-            uint32_t *mrow = mrow0;
+            unsigned mkeep = 0u;                          // lane r: word 0 of row r; lane 16 + r: word 1
             e = zero4();
             dprod = make_float2(1.f, 1.f);
 #pragma unroll
@@ -685,11 +691,14 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
                     const unsigned bits = ((oA ? 1u : 0u) | (oB ? 2u : 0u)) << (2 * (lane & 15));
                     const unsigned w0 = __reduce_or_sync(0xffffffffu, lane < 16 ? bits : 0u);
                     const unsigned w1 = __reduce_or_sync(0xffffffffu, lane < 16 ? 0u : bits);
-                    if (FULL || i < nvalid) {
-                        if (lane == 0) mrow[0] = w0;
-                        if (lane == 16 && second_word) mrow[1] = w1;
+                    // rows are parked in lanes and stored sixteen at a time
+                    if (lane == (i & 15)) mkeep = w0;
+                    if (lane == 16 + (i & 15)) mkeep = w1;
+                    if ((i & 15) == 15 || i == T - 1) {
+                        const int r = i - (i & 15) + (lane & 15);
+                        if ((lane & 15) <= (i & 15) && (FULL || r < nvalid) && (lane < 16 || second_word))
+                            mrow0[(long long)r * prm.MW + (lane >> 4)] = mkeep;
                     }
-                    mrow += prm.MW;
                 }
                 if (FULL || i < nvalid) {
                     if constexpr (DYN) {
@@ -707,9 +716,12 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
         };
         using yes = std::true_type;
         using no = std::false_type;
-        const float nearest = want_mask ? pass(no{}, yes{}) : pass(no{}, no{});
+        float nearest;
+        if constexpr (MASKED) nearest = want_mask ? pass(no{}, yes{}) : pass(no{}, no{});
+        else nearest = pass(no{}, no{});
         if (__any_sync(0xffffffffu, nearest <= hw)) {
-            if (want_mask) pass(yes{}, yes{}); else pass(yes{}, no{});
+            if constexpr (MASKED) { if (want_mask) pass(yes{}, yes{}); else pass(yes{}, no{}); }
+            else pass(yes{}, no{});
         }
     } else {
         if (early_ptr != nullptr) {
@@ -1146,7 +1158,7 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
     }
 }
 
-template <int T, int W, int KIND, bool VEC, int MINB, bool DYN = false, bool EAR = false, int IO = IO_F32>
+template <int T, int W, int KIND, bool VEC, int MINB, bool DYN = false, bool EAR = false, int IO = IO_F32, bool MASKED = true>
 __global__ void __launch_bounds__(W * 32, MINB) cawn_scan_kernel(const ScanParams prm)
 {
     constexpr int TILE = T * W;
@@ -1159,8 +1171,8 @@ __global__ void __launch_bounds__(W * 32, MINB) cawn_scan_kernel(const ScanParam
     const int k = blockIdx.z;                         // tile index along (logical) time
     grid_launch_dependents();
     const bool full = ((long long)(k + 1) * TILE <= prm.L) && (g * 64 + 64 <= prm.C);
-    if (full) scan_tile<T, W, KIND, VEC, DYN, true, EAR, IO>(prm, sm, g, b, k);
-    else      scan_tile<T, W, KIND, VEC, DYN, false, EAR, IO>(prm, sm, g, b, k);
+    if (full) scan_tile<T, W, KIND, VEC, DYN, true, EAR, IO, MASKED>(prm, sm, g, b, k);
+    else      scan_tile<T, W, KIND, VEC, DYN, false, EAR, IO, MASKED>(prm, sm, g, b, k);
 }
 
 }  // namespace cawn
