@@ -32,7 +32,7 @@ BYTES_PER_ELEMENT = 16         # algorithmic: read one complex64 push, write one
 # workload, from the ncu capture summarised in profiles/cawn_scan_fwd_cfg1_ncu.md: 101.4 MB read
 # + 47.4 MB written while an isolated launch runs (the rest of its 100.7 MB of output is still
 # dirty in L2 when it ends).  Set to None whenever the kernel changes after the capture.
-NCU_DRAM_BYTES_PER_LAUNCH = 148914688
+NCU_DRAM_BYTES_PER_LAUNCH = 148325120
 
 
 def workload():
@@ -279,7 +279,7 @@ def run_ours(args):
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                          "frac": achieved / peak, "peak_kind": peak_kind + " copy bandwidth",
                          "frac_of_nominal_8000": achieved / 8000.0,
-                         "kernel": "cawn_scan_kernel<16,8,KIND_FWD,VEC,3>", "kernel_ms": kernel_ms,
+                         "kernel": "cawn_scan_kernel<16,8,KIND_FWD,VEC,3> (no mask output)", "kernel_ms": kernel_ms,
                          "algorithmic_bytes_per_launch": nelem * BYTES_PER_ELEMENT,
                          "traffic": NCU_DRAM_BYTES_PER_LAUNCH},
             "e2e": {"value": whole_job_value(world, tokens, e2e_ms), "unit": UNIT,
