@@ -421,6 +421,20 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
         cp_async_commit();
     }
 
+    // Fused path: this lane's conv taps (right-aligned: taps the conv does not have are zero) and
+    // bias, requested here so that they arrive while the tile is still in flight.
+    float wA[4] = {}, wB[4] = {}, bA = 0.f, bB = 0.f;
+    if constexpr (KIND == KIND_FUSED) {
+        const int Kc = prm.conv_k;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int kk = j - (4 - Kc);
+            if (kk >= 0 && vA) wA[j] = prm.conv_w[(long long)c0 * Kc + kk];
+            if (kk >= 0 && vB) wB[j] = prm.conv_w[(long long)(c0 + 1) * Kc + kk];
+        }
+        if (prm.conv_bias != nullptr) { if (vA) bA = prm.conv_bias[c0]; if (vB) bB = prm.conv_bias[c0 + 1]; }
+    }
+
     // ---- per-channel coefficients, in double, rounded once --------------------------------
     // Three independent tasks per channel, one thread each: a^n = gamma^n (cos n theta, sin n theta)
     // for n = 1, T, TILE.  n theta is exact in double (theta is a float, n a small integer).
@@ -547,15 +561,6 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
             er1 = ld_record(early_ptr + 2 * lane + 1);
         }
         const int Kc = prm.conv_k;
-        float wA[4], wB[4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const int kk = j - (4 - Kc);
-            wA[j] = (kk >= 0 && vA) ? prm.conv_w[(long long)c0 * Kc + kk] : 0.f;
-            wB[j] = (kk >= 0 && vB) ? prm.conv_w[(long long)(c0 + 1) * Kc + kk] : 0.f;
-        }
-        const float bA = (prm.conv_bias != nullptr && vA) ? prm.conv_bias[c0] : 0.f;
-        const float bB = (prm.conv_bias != nullptr && vB) ? prm.conv_bias[c0 + 1] : 0.f;
         __syncthreads();                 // every thread holds its hidden rows: the staging area may go
         const bool act = prm.clamp_silu != 0;
         const float tau = prm.gate_tau;
@@ -759,6 +764,18 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
                 if (FULL || i < nvalid) e = cfma2(a, e, xs[i * 32]);
         }
     }
+    // MIXBWD: conv taps and bias for phase 3, requested here so that they arrive during the carry exchange
+    float mwA[4] = {}, mwB[4] = {}, mbA = 0.f, mbB = 0.f;
+    if constexpr (MIX) {
+        const int Kc = prm.conv_k;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int kk = j - (4 - Kc);
+            if (kk >= 0 && vA) mwA[j] = prm.conv_w[(long long)c0 * Kc + kk];
+            if (kk >= 0 && vB) mwB[j] = prm.conv_w[(long long)(c0 + 1) * Kc + kk];
+        }
+        if (prm.conv_bias != nullptr) { if (vA) mbA = prm.conv_bias[c0]; if (vB) mbB = prm.conv_bias[c0 + 1]; }
+    }
     sm.sE[w][lane] = e;
     if constexpr (DYN) sm.sD[w][lane] = dprod;
     if (tid == 0 && arrived == gridDim.x * gridDim.y * gridDim.z - 1) {
@@ -913,19 +930,10 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
         if constexpr (DYN && REV) gstep = gfirst;
         // MIXBWD: conv taps (right-aligned: tap j multiplies the hidden row 3 - j steps back), the
         // rolling window of hidden rows, and the sums for the conv gradients
-        float mwA[4] = {}, mwB[4] = {}, mbA = 0.f, mbB = 0.f;
         float2 hwin[4] = {};                             // h(t), h(t-1), h(t-2), h(t-3) of the current row
         float caA[5] = {}, caB[5] = {};
         const bool mact = prm.clamp_silu != 0;
         if constexpr (MIX) {
-            const int Kc = prm.conv_k;
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const int kk = j - (4 - Kc);
-                mwA[j] = (kk >= 0 && vA) ? prm.conv_w[(long long)c0 * Kc + kk] : 0.f;
-                mwB[j] = (kk >= 0 && vB) ? prm.conv_w[(long long)(c0 + 1) * Kc + kk] : 0.f;
-            }
-            if (prm.conv_bias != nullptr) { if (vA) mbA = prm.conv_bias[c0]; if (vB) mbB = prm.conv_bias[c0 + 1]; }
 #pragma unroll
             for (int r = 0; r < 3; ++r) hwin[r + 1] = *reinterpret_cast<const float2 *>(&sm.hrev[w * T + r][2 * lane]);
         }
