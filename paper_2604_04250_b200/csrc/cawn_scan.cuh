@@ -928,6 +928,14 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
         // the row processed before it), and the running sum of the logit gradient
         float2 gstep = make_float2(0.f, 0.f), sacc = make_float2(0.f, 0.f);
         if constexpr (DYN && REV) gstep = gfirst;
+        // DYN backward: the heads this 64-channel group touches
+        int h_lo = 0, h_hi = 0;
+        if constexpr (DYN && REV) {
+            const int c_hi = g * 64 + 63 < C - 1 ? g * 64 + 63 : C - 1;
+            h_lo = (g * 64) / prm.F;
+            h_hi = c_hi / prm.F;
+        }
+        float rowsum[DYN && REV ? T : 1] = {};           // per row: this lane's share of the head's logit gradient
         // MIXBWD: conv taps (right-aligned: tap j multiplies the hidden row 3 - j steps back), the
         // rolling window of hidden rows, and the sums for the conv gradients
         float2 hwin[4] = {};                             // h(t), h(t-1), h(t-2), h(t-3) of the current row
@@ -984,11 +992,10 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
                             const float sA = gown.x * (1.f - gown.x) * fmaf(a.x, uAx, a.y * uAy);
                             const float sB = gown.y * (1.f - gown.y) * fmaf(a.z, uBx, a.w * uBy);
                             sacc.x += sA; sacc.y += sB;
-                            if (prm.grad_logit != nullptr) {
+                            if (prm.grad_logit != nullptr && h_lo == h_hi) {
+                                rowsum[i] = sA + sB;             // one head: all rows are reduced together below
+                            } else if (prm.grad_logit != nullptr) {
                                 // sum over the harmonics of each head present in this 64-channel group
-                                const int h_lo = (g * 64) / prm.F;
-                                const int c_hi = g * 64 + 63 < C - 1 ? g * 64 + 63 : C - 1;
-                                const int h_hi = c_hi / prm.F;
                                 for (int h = h_lo; h <= h_hi; ++h) {
                                     float v = (vA && hA == h ? sA : 0.f) + (vB && hB == h ? sB : 0.f);
 #pragma unroll
@@ -1032,6 +1039,29 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
             for (int i = 0; i < T; ++i) step_row(i, false);
         }
         sacc_out = sacc;
+        if constexpr (DYN && REV) {
+            if (prm.grad_logit != nullptr && prm.aux != nullptr && h_lo == h_hi) {
+                // T row sums over the 32 lanes at once: each exchange halves the rows a lane still
+                // carries, so that after log2(T) rounds lane (32/T) r holds row r's partial; then
+                // plain butterflies among the 32/T lanes that share a row.  9 shuffles for 8 rows.
+#pragma unroll
+                for (int n = T / 2, off = 16; n >= 1; n >>= 1, off >>= 1) {
+                    const bool upper = (lane & off) != 0;
+#pragma unroll
+                    for (int j = 0; j < n; ++j) {
+                        const float send = upper ? rowsum[j] : rowsum[j + n];
+                        const float keep = upper ? rowsum[j + n] : rowsum[j];
+                        rowsum[j] = keep + __shfl_xor_sync(0xffffffffu, send, off);
+                    }
+                }
+#pragma unroll
+                for (int off = 16 / T; off >= 1; off >>= 1) rowsum[0] += __shfl_xor_sync(0xffffffffu, rowsum[0], off);
+                constexpr int LPR = 32 / T;              // lanes per row
+                const int row = lane / LPR;
+                if (lane % LPR == 0 && (FULL || row < nvalid))
+                    atomicAdd(prm.grad_logit + ((long long)b * L + (t_first - row)) * prm.H + h_lo, rowsum[0]);
+            }
+        }
         // An Inf or NaN that entered anywhere (an input, the carried state, an overflow) is still
         // in the chain's last state: the recurrence never makes it finite again.  (A NaN push
         // itself fails the gate's comparison and is dropped like any closed gate.)
