@@ -151,7 +151,9 @@ CAWN_API int cawn_workspace_init(void *workspace, size_t workspace_bytes, void *
  *               gate, z = m (cos, sin)(phase).
  * gamma/theta:  [C] device.  With CAWN_FLAG_RETENTION_DYNAMIC gamma is ignored and
  *               gamma_logit [B,L,H], freq_bias [F] (device) define the retention
- *               (Section "Multi-Head Dynamic Parameter Projection", item 4).
+ *               (Section "Multi-Head Dynamic Parameter Projection", item 4); available for
+ *               both input forms (with conv_k >= 1 this is the paper's own layer: Temporal
+ *               Syntax Cache, gated push and per-token retention in one pass).
  * state_in:     state blob (device) or NULL for a zero state.
  * y:            [B,L,C] complex64 (device), clamped if clamp_abs > 0.
  * state_out:    state blob (device) or NULL.  May alias state_in.

@@ -235,10 +235,11 @@ def forward(p, gamma, theta, gate_eps, state_in=None, clamp_abs=0.0, **kw):
 
 
 def fused_forward(h, w, gamma, theta, gate_eps, gate_tau, bias=None,
-                  clamp_silu=False, tail_in=None, state_in=None, clamp_abs=0.0):
-    """prelude -> scan on fp32 hidden states.  Returns (y, state_out, mask, tail_out)."""
+                  clamp_silu=False, tail_in=None, state_in=None, clamp_abs=0.0, **kw):
+    """prelude -> scan on fp32 hidden states.  Returns (y, state_out, mask, tail_out).
+    ``gamma=None`` with ``gamma_logit=, freq_bias=, H=`` gives the time-varying retention."""
     z, mask, tail = prelude(h, w, bias, clamp_silu, tail_in, gate_eps, gate_tau)
-    y, so = scan(z, theta, gamma=gamma, state_in=state_in, clamp_abs=clamp_abs)
+    y, so = scan(z, theta, gamma=gamma, state_in=state_in, clamp_abs=clamp_abs, **kw)
     return y, so, mask, tail
 
 

@@ -211,6 +211,16 @@ def _cfg4(args, cb, inputs, dev, IND):
                max(args.steps // 2, 5), args.warmup)
     assert cb.cawn_poll_status(ws) == 0
     _report("cfg4_fused" if B == cfg.B else "cfg4_fused_B%d" % B, B * L, B * L * C * 12, ms, 1)
+    if "dynamic" in args.only or not args.only:
+        dd = inputs.dynamic_retention_inputs(B, L, cfg.H, cfg.F, 7)
+        gl, fb = dev(dd["gamma_logit"]), dev(dd["freq_bias"])
+        prm_d = cb.make_params(B, L, cfg.H, cfg.F, gate_eps=cfg.gate_eps, gate_tau=float(inputs.gate_tau(cfg.gate_eps)),
+                               conv_k=cfg.conv_k, flags=IND | cb.CAWN_FLAG_RETENTION_DYNAMIC)
+        ms = _time(lambda i: cb.cawn_phase_accumulate_fwd(prm_d, hs[i % NS], None, t, ys[i % NS], ws, conv_w=w,
+                                                          gamma_logit=gl, freq_bias=fb),
+                   max(args.steps // 2, 5), args.warmup)
+        assert cb.cawn_poll_status(ws) == 0
+        _report("cfg4_fused_dynamic_retention", B * L, B * L * (C * 12 + cfg.H * 4), ms, 1)
     if "bf16" in args.only or not args.only:
         prm16 = cb.make_params(B, L, cfg.H, cfg.F, gate_eps=cfg.gate_eps, gate_tau=float(inputs.gate_tau(cfg.gate_eps)),
                                conv_k=cfg.conv_k, flags=IND | cb.CAWN_FLAG_INPUT_BF16 | cb.CAWN_FLAG_OUTPUT_BF16)

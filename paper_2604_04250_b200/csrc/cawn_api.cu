@@ -137,8 +137,9 @@ inline cudaError_t launch_fwd(TileShape ts, const ScanParams &sp, cudaStream_t s
     if (sp.ear_w != nullptr) return launch_fwd_ear(ts, sp, st);
     return dyn ? launch_fwd_dynamic(ts, sp, st) : launch_fwd_static(ts, sp, st);
 }
-inline cudaError_t launch_fused(TileShape ts, const ScanParams &sp, cudaStream_t st, int io = 0)
+inline cudaError_t launch_fused(TileShape ts, const ScanParams &sp, cudaStream_t st, int io = 0, bool dyn = false)
 {
+    if (dyn) return launch_fused_dynamic(ts, sp, st);
     if (io != 0) return launch_fused_bf16(ts, sp, st, io);
     return sp.ear_w != nullptr ? launch_fused_ear(ts, sp, st) : launch_fused_plain(ts, sp, st);
 }
@@ -300,7 +301,6 @@ static int fwd_common(const cawn_params *params, const void *input,
         if (!aligned(ear_w, 4) || !aligned(ear_bias, 4)) return CAWN_ERR_MISALIGNED;
     }
     if (dyn) {
-        if (fused) return CAWN_ERR_UNSUPPORTED;
         if (gamma_logit == nullptr || freq_bias == nullptr) return CAWN_ERR_NULL_POINTER;
         if (!aligned(gamma_logit, 4) || !aligned(freq_bias, 4)) return CAWN_ERR_MISALIGNED;
     }
@@ -361,7 +361,8 @@ static int fwd_common(const cawn_params *params, const void *input,
             sp.tail_in = state_in ? reinterpret_cast<const float *>(reinterpret_cast<const char *>(state_in) + tail_off) : nullptr;
             sp.tail_out = state_out ? reinterpret_cast<float *>(reinterpret_cast<char *>(state_out) + tail_off) : nullptr;
         }
-        if (launch_fused(ts, sp, st, io) != cudaSuccess) return CAWN_ERR_CUDA;
+        sp.gamma_logit = gamma_logit; sp.freq_bias = freq_bias;
+        if (launch_fused(ts, sp, st, io, dyn) != cudaSuccess) return CAWN_ERR_CUDA;
         return CAWN_OK;
     }
     sp.gamma_logit = gamma_logit; sp.freq_bias = freq_bias; sp.H = params->H; sp.F = params->F;

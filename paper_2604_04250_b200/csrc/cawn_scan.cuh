@@ -268,7 +268,6 @@ template <int T, int W, int KIND, bool VEC, bool DYN, bool FULL, bool EAR = fals
 __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, KIND, DYN> &sm,
                                           const int g, const int b, const int k)
 {
-    static_assert(!(DYN && KIND == KIND_FUSED), "time-varying retention is not built for the fused path");
     static_assert(!(EAR && (DYN || kind_is_bwd(KIND))), "the Ear epilogue belongs to the static forward");
     static_assert(IO == IO_F32 || (!EAR && !DYN && !kind_is_bwd(KIND)), "bf16 storage is built for the static forward");
     constexpr bool IN16 = (IO & IO_IN_BF16) != 0, OUT16 = (IO & IO_OUT_BF16) != 0;
@@ -578,6 +577,19 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
         const float2 ar2 = make_float2(a.x, a.z), ai2 = make_float2(a.y, a.w), nai2 = make_float2(-a.y, -a.w);
         const float2 one2 = make_float2(1.f, 1.f);
         float2 er2 = make_float2(0.f, 0.f), ei2 = er2;
+        // DYN: the rows' retention logits, all requested up front so that their latencies overlap
+        float2 lgf[DYN ? T : 1];
+        if constexpr (DYN) {
+#pragma unroll
+            for (int i = 0; i < T; ++i) {
+                lgf[i] = make_float2(0.f, 0.f);
+                if (FULL || i < nvalid) {
+                    const float *gl = prm.gamma_logit + ((long long)b * L + s0 + i) * prm.H;
+                    if (vA) lgf[i].x = gl[hA];
+                    if (vB) lgf[i].y = gl[hB];
+                }
+            }
+        }
 #pragma unroll
         for (int i = 0; i < T; ++i) {
             float2 u = b2;
@@ -624,9 +636,20 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
                 }
             }
             if (FULL || i < nvalid) {
-                const float2 nr = __ffma2_rn(ar2, er2, __ffma2_rn(nai2, ei2, zr));
-                const float2 ni = __ffma2_rn(ar2, ei2, __ffma2_rn(ai2, er2, zi));
-                er2 = nr; ei2 = ni;
+                if constexpr (DYN) {
+                    // e <- gamma_t (a e) + z, the factor pair kept for phase 3
+                    const float2 gm = make_float2(vA ? sigmoidf_fast(lgf[i].x + fbA) : 0.f,
+                                                  vB ? sigmoidf_fast(lgf[i].y + fbB) : 0.f);
+                    sm.sG[w * T + i][lane] = gm;
+                    dprod.x *= gm.x; dprod.y *= gm.y;
+                    const float2 tr = __ffma2_rn(ar2, er2, __fmul2_rn(nai2, ei2));
+                    const float2 ti = __ffma2_rn(ar2, ei2, __fmul2_rn(ai2, er2));
+                    er2 = __ffma2_rn(gm, tr, zr); ei2 = __ffma2_rn(gm, ti, zi);
+                } else {
+                    const float2 nr = __ffma2_rn(ar2, er2, __ffma2_rn(nai2, ei2, zr));
+                    const float2 ni = __ffma2_rn(ar2, ei2, __ffma2_rn(ai2, er2, zi));
+                    er2 = nr; ei2 = ni;
+                }
             }
         }
         e = make_float4(er2.x, ei2.x, er2.y, ei2.y);
@@ -1022,9 +1045,17 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
             for (int i = 0; i < T; ++i) {
                 if (FULL || i < nvalid) {
                     const float4 z = xs[i * 32];
-                    const float2 nr = __ffma2_rn(ar2, Pr, __ffma2_rn(nai2, Pi, make_float2(z.x, z.y)));
-                    const float2 ni = __ffma2_rn(ar2, Pi, __ffma2_rn(ai2, Pr, make_float2(z.z, z.w)));
-                    Pr = nr; Pi = ni;
+                    if constexpr (DYN) {
+                        gstep = sm.sG[w * T + i][lane];
+                        const float2 tr = __ffma2_rn(ar2, Pr, __fmul2_rn(nai2, Pi));
+                        const float2 ti = __ffma2_rn(ar2, Pi, __fmul2_rn(ai2, Pr));
+                        Pr = __ffma2_rn(gstep, tr, make_float2(z.x, z.y));
+                        Pi = __ffma2_rn(gstep, ti, make_float2(z.z, z.w));
+                    } else {
+                        const float2 nr = __ffma2_rn(ar2, Pr, __ffma2_rn(nai2, Pi, make_float2(z.x, z.y)));
+                        const float2 ni = __ffma2_rn(ar2, Pi, __ffma2_rn(ai2, Pr, make_float2(z.z, z.w)));
+                        Pr = nr; Pi = ni;
+                    }
                     float4 o = make_float4(Pr.x, Pi.x, Pr.y, Pi.y);
                     if (cl > 0.f) o = clamp4(o, cl);
                     store_row(i, o);

@@ -105,3 +105,45 @@ def test_dynamic_backward_shapes(B, L, H, F, saved_kind):
     for k in ("dgamma_logit", "dfreq_bias", "dtheta"):
         assert not np.isnan(got[k]).any(), k
         assert floored_rel_err(got[k], ref[k]) < TOL, k
+
+
+@pytest.mark.parametrize("B,L,H,F,Kc", [(1, 3, 1, 64, 4), (2, 200, 2, 64, 4), (1, 333, 3, 32, 3), (2, 150, 5, 16, 4),
+                                        (1, 131, 3, 11, 4), (1, 515, 12, 64, 4), (2, 20, 2, 64, 2)])
+def test_fused_path_with_dynamic_retention(B, L, H, F, Kc):
+    """The paper's own combination: conv prelude and gated push feeding a recurrence whose retention
+    varies per token and head; chunked in two calls with the state blob carried."""
+    import torch
+    from gpu_util import dev, state_blob, split_blob
+    from paper_2604_04250_b200 import binding as cb
+    C = H * F
+    d = inputs.fused_inputs(B, L, C, 700 + L, conv_k=Kc, with_tail=True)
+    d.update(inputs.dynamic_retention_inputs(B, L, H, F, 701 + L))
+    eps, tau = 0.1, float(inputs.gate_tau(0.1))
+    rng = np.random.default_rng(9)
+    P_in = (rng.normal(0, 2, (B, C)) + 1j * rng.normal(0, 2, (B, C))).astype(np.complex64)
+    y_ref, so_ref, m_ref, tail_ref = oracle.fused_forward(
+        d["h"], d["conv_w"], None, d["theta"], eps, tau, bias=d.get("conv_bias"), tail_in=d["tail_in"],
+        state_in=P_in.astype(np.complex128), gamma_logit=d["gamma_logit"], freq_bias=d["freq_bias"], H=H)
+    blob, off = state_blob(B, C, Kc, P_in, d["tail_in"])
+    t, w, bias = dev(d["theta"]), dev(d["conv_w"]), dev(d.get("conv_bias"))
+    fb = dev(d["freq_bias"])
+    y = torch.full((B, L, C), float("nan"), dtype=torch.complex64, device="cuda")
+    m = torch.zeros((B, L, (C + 31) // 32), dtype=torch.int32, device="cuda")
+    cut = L // 2
+    for lo, hi in ((0, cut), (cut, L)):
+        n = hi - lo
+        prm = cb.make_params(B, n, H, F, gate_eps=eps, gate_tau=tau, conv_k=Kc, flags=cb.CAWN_FLAG_RETENTION_DYNAMIC)
+        ws = cb.new_workspace(prm, cb.CAWN_OP_FWD)
+        yy = torch.full((B, n, C), float("nan"), dtype=torch.complex64, device="cuda")
+        mm = torch.zeros((B, n, (C + 31) // 32), dtype=torch.int32, device="cuda")
+        cb.cawn_phase_accumulate_fwd(prm, dev(d["h"][:, lo:hi]), None, t, yy, ws, conv_w=w, conv_bias=bias,
+                                     gamma_logit=dev(d["gamma_logit"][:, lo:hi]), freq_bias=fb,
+                                     state_in=blob, state_out=blob, gate_mask=mm)
+        assert cb.cawn_poll_status(ws) == 0
+        y[:, lo:hi] = yy
+        m[:, lo:hi] = mm
+    assert floored_rel_err(y.cpu().numpy(), y_ref) < TOL
+    P_out, tail_out = split_blob(blob, off, B, C, Kc)
+    assert floored_rel_err(P_out, so_ref) < TOL
+    assert np.array_equal(tail_out, tail_ref.astype(np.float32))
+    assert np.array_equal(unpack_mask(m.cpu().numpy().view(np.uint32), C), m_ref)
