@@ -281,6 +281,16 @@ def _cfg2(args, cb, inputs, dev, IND):
     assert cb.cawn_poll_status(ws) == 0
     _report("cfg2_chunked_prefill", ncalls * n, ncalls * n * C * 16, ms, ncalls,
             {"us_per_4096_token_call": ms * 1e3 / ncalls, "note": "one launch per chunk, state carried on the device"})
+    # the same 64 calls recorded once into a CUDA graph: takes the host's per-call cost out
+    side = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        prefill(0)
+    ms = _time(lambda i: graph.replay(), max(args.steps // 10, 3), 2)
+    assert cb.cawn_poll_status(ws) == 0
+    _report("cfg2_chunked_prefill_cuda_graph", ncalls * n, ncalls * n * C * 16, ms, ncalls,
+            {"us_per_4096_token_call": ms * 1e3 / ncalls, "note": "64 chunk calls replayed from one CUDA graph"})
 
 
 if __name__ == "__main__":

@@ -192,6 +192,21 @@ def test_host_buffer_entry_point_sliced(B, L, C):
         assert np.array_equal(unpack_mask(m.numpy().view(np.uint32), C), m_ref)
 
 
+@pytest.mark.parametrize("B,L,C", [(1, 1153, 64), (1, 1920, 128), (2, 2048, 64), (1, 2049, 192), (1, 4096, 768), (3, 3000, 100),
+                                   (1, 8 * 128 + 1, 64), (1, 16 * 128, 64), (1, 17 * 128 + 5, 64), (1, 31 * 128, 64)])
+def test_lengths_around_checkpoint_tiles(B, L, C):
+    """Lengths on both sides of one, two and four checkpoint tiles (every seventh tile of 128 steps
+    publishes its carry-in), with a carried state and no mask; twice, bit for bit."""
+    from gpu_util import run_fwd
+    d = inputs.scan_inputs(B, L, C, seed=170 + L % 97, with_state=True)
+    y, so, _ = run_fwd(d["p"], d["gamma"], d["theta"], 0.1, state_in=d["state_in"], want_mask=False)
+    y_ref, so_ref, _ = oracle.forward(d["p"], d["gamma"], d["theta"], 0.1, state_in=d["state_in"].astype(np.complex128))
+    assert floored_rel_err(y, y_ref, axes=(0, 1)) < TOL
+    assert floored_rel_err(so, so_ref) < TOL
+    y2, so2, _ = run_fwd(d["p"], d["gamma"], d["theta"], 0.1, state_in=d["state_in"], want_mask=False)
+    assert np.array_equal(y.view(np.uint32), y2.view(np.uint32)) and np.array_equal(so.view(np.uint32), so2.view(np.uint32))
+
+
 def test_repeatable_bitwise():
     from gpu_util import run_fwd
     d = inputs.scan_inputs(4, 2048, 256, seed=16)
