@@ -254,6 +254,25 @@ CAWN_API int cawn_mixing_bwd(const cawn_params *params,
                              void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
+ * cawn_mixing_bwd with the paper's time-varying retention (the fused path run with
+ * CAWN_FLAG_RETENTION_DYNAMIC, which params->flags must carry): the backward of the whole
+ * Resonance mixing step as the paper defines it — Temporal Syntax Cache, gated push, per-token
+ * per-head retention (Section "Multi-Head Dynamic Parameter Projection").  gamma_logit [B,L,H],
+ * freq_bias [F] replace gamma; grad_gamma_logit [B,L,H] (zeroed by the call, then accumulated
+ * with atomic adds) and grad_freq_bias [F] replace grad_gamma; each may be NULL.  Everything
+ * else as cawn_mixing_bwd, including the workspace size.
+ */
+CAWN_API int cawn_mixing_bwd_dynamic(const cawn_params *params,
+                                     const float *h, const float *conv_w, const float *conv_bias,
+                                     const float *gamma_logit, const float *freq_bias, const float *theta,
+                                     const void *saved_states, const void *state_in,
+                                     const void *grad_y, const void *grad_state_out,
+                                     float *grad_h, float *grad_conv_w, float *grad_conv_bias,
+                                     float *grad_gamma_logit, float *grad_freq_bias, float *grad_theta,
+                                     void *grad_state_in,
+                                     void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
  * Forward with the front of the Convolutional SwiGLU Ear as the scan's epilogue (Eq. (wave_synth)
  * and Section "Projection to Hidden State: The Convolutional SwiGLU Ear", the depth-wise 1-D
  * convolution across the K harmonics).  Everything up to the clamped state y_t is

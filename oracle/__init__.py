@@ -268,9 +268,10 @@ def prelude_bwd(h, w, dz, bias=None, clamp_silu=False, tail_in=None, gate_eps=0.
 
 
 def fused_backward(h, w, gamma, theta, G, gate_eps, gate_tau, bias=None, clamp_silu=False, tail_in=None,
-                   state_in=None, dstate_out=None, dtail_out=None):
-    """prelude -> scan forward, then scan_bwd -> prelude_bwd.  Returns the union of both dicts."""
+                   state_in=None, dstate_out=None, dtail_out=None, **kw):
+    """prelude -> scan forward, then scan_bwd -> prelude_bwd.  Returns the union of both dicts.
+    ``gamma=None`` with ``gamma_logit=, freq_bias=, H=`` gives the time-varying retention."""
     z, mask, _ = prelude(h, w, bias, clamp_silu, tail_in, gate_eps, gate_tau)
-    out = scan_bwd(z, theta, G, gamma=gamma, state_in=state_in, dstate_out=dstate_out)
+    out = scan_bwd(z, theta, G, gamma=gamma, state_in=state_in, dstate_out=dstate_out, **kw)
     out.update(prelude_bwd(h, w, out["dp"], bias, clamp_silu, tail_in, gate_eps, gate_tau, dtail_out))
     return out

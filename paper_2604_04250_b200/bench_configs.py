@@ -257,6 +257,19 @@ def _cfg4_bwd(args, cb, inputs, dev):
     # reads grad_y (8) + P (8) + h (4), writes grad_h (4)
     _report("cfg4_mixing_bwd" if B == cfg.B else "cfg4_mixing_bwd_B%d" % B, B * L, B * L * C * 24, ms, 4,
             {"note": "reverse scan with the prelude backward as its epilogue, seam rows, two reductions"})
+    # the same with time-varying retention (the paper's layer form)
+    dd = inputs.dynamic_retention_inputs(B, L, cfg.H, cfg.F, 7)
+    gl, fb = dev(dd["gamma_logit"]), dev(dd["freq_bias"])
+    prm_d = cb.make_params(B, L, cfg.H, cfg.F, gate_eps=cfg.gate_eps, gate_tau=float(inputs.gate_tau(cfg.gate_eps)),
+                           conv_k=cfg.conv_k, flags=cb.CAWN_FLAG_RETENTION_DYNAMIC)
+    cb.cawn_phase_accumulate_fwd(prm_d, h, None, t, P, wf, conv_w=w, gamma_logit=gl, freq_bias=fb)
+    ggl, gfb = torch.empty((B, L, cfg.H), device="cuda"), torch.empty(cfg.F, device="cuda")
+    ms = _time(lambda i: cb.cawn_mixing_bwd_dynamic(prm_d, h, w, gl, fb, t, gy, gh, wb, saved_states=P, grad_conv_w=gw,
+                                                    grad_conv_bias=gb, grad_gamma_logit=ggl, grad_freq_bias=gfb, grad_theta=gt),
+               max(args.steps // 2, 5), args.warmup)
+    assert cb.cawn_poll_status(wb) == 0
+    _report("cfg4_mixing_bwd_dynamic_retention" if B == cfg.B else "cfg4_mixing_bwd_dynamic_retention_B%d" % B, B * L,
+            B * L * (C * 24 + cfg.H * 8), ms, 6, {"note": "plus the memset of the logit gradient and the frequency-bias reduction"})
 
 
 def _cfg2(args, cb, inputs, dev, IND):

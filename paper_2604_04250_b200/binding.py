@@ -39,7 +39,7 @@ EXPORTS = (
     "cawn_phase_accumulate_fwd", "cawn_phase_accumulate_bwd", "cawn_state_carry",
     "cawn_poll_status", "cawn_phase_accumulate_fwd_host", "cawn_phase_accumulate_fwd_static",
     "cawn_phase_accumulate_bwd_dynamic", "cawn_mixing_bwd", "cawn_phase_accumulate_fwd_ear",
-    "cawn_workspace_set_wait_hook",
+    "cawn_workspace_set_wait_hook", "cawn_mixing_bwd_dynamic",
 )
 
 
@@ -88,6 +88,7 @@ def lib():
         L.cawn_phase_accumulate_bwd_dynamic.argtypes = [pp, vp, ctypes.c_int, fp, fp, fp, vp, vp, vp, vp, fp, fp, fp, vp, vp, sz, vp]
         L.cawn_mixing_bwd.argtypes = [pp, fp, fp, fp, fp, fp, vp, vp, vp, vp, fp, fp, fp, fp, fp, vp, vp, sz, vp]
         L.cawn_phase_accumulate_fwd_ear.argtypes = [pp, vp, fp, fp, fp, fp, vp, fp, fp, ctypes.c_int, fp, vp, vp, vp, sz, vp]
+        L.cawn_mixing_bwd_dynamic.argtypes = [pp, fp, fp, fp, fp, fp, fp, vp, vp, vp, vp, fp, fp, fp, fp, fp, fp, vp, vp, sz, vp]
         L.cawn_state_carry.argtypes = [pp, vp, vp, ctypes.c_int64, fp, fp, vp, vp]
         L.cawn_poll_status.argtypes = [vp, vp]
         L.cawn_workspace_set_wait_hook.argtypes = [vp, ctypes.c_int, ctypes.c_uint, vp]
@@ -179,6 +180,16 @@ def cawn_phase_accumulate_bwd(params, saved, saved_kind, gamma, theta, grad_y, g
         _dp(grad_y), _dp(grad_state_out), _dp(grad_p), _dp(grad_gamma), _dp(grad_theta),
         _dp(grad_state_in), _dp(workspace), workspace.numel() * workspace.element_size(),
         _stream(stream)), "cawn_phase_accumulate_bwd")
+
+
+def cawn_mixing_bwd_dynamic(params, h, conv_w, gamma_logit, freq_bias, theta, grad_y, grad_h, workspace, conv_bias=None,
+                            saved_states=None, state_in=None, grad_state_out=None, grad_conv_w=None, grad_conv_bias=None,
+                            grad_gamma_logit=None, grad_freq_bias=None, grad_theta=None, grad_state_in=None, stream=None):
+    _check(lib().cawn_mixing_bwd_dynamic(
+        ctypes.byref(params), _dp(h), _dp(conv_w), _dp(conv_bias), _dp(gamma_logit), _dp(freq_bias), _dp(theta),
+        _dp(saved_states), _dp(state_in), _dp(grad_y), _dp(grad_state_out), _dp(grad_h), _dp(grad_conv_w),
+        _dp(grad_conv_bias), _dp(grad_gamma_logit), _dp(grad_freq_bias), _dp(grad_theta), _dp(grad_state_in),
+        _dp(workspace), workspace.numel() * workspace.element_size(), _stream(stream)), "cawn_mixing_bwd_dynamic")
 
 
 def cawn_state_carry(params, state_prev, state_local, n_steps, gamma, theta, state_out, stream=None):

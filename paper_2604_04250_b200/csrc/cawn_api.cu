@@ -151,7 +151,7 @@ inline cudaError_t launch_bwd(TileShape ts, const ScanParams &sp, cudaStream_t s
 // Workspace of cawn_mixing_bwd: header, carry records, per-tile sums for grad_gamma / grad_theta,
 // du at the tile seams, per-tile sums for the conv gradients.
 struct MixBwdLayout {
-    size_t off_rec, off_qpart, off_edge, off_cpart, total;
+    size_t off_rec, off_qpart, off_spart, off_edge, off_cpart, total;
 };
 MixBwdLayout mix_bwd_layout(const cawn_params *p)
 {
@@ -161,6 +161,7 @@ MixBwdLayout mix_bwd_layout(const cawn_params *p)
     size_t o = sizeof(WsHeader);
     m.off_rec = o;    o += round_up(g.rec_bytes, 256);
     m.off_qpart = o;  o += round_up(tiles * g.C * sizeof(float2), 256);
+    m.off_spart = o;  o += round_up(tiles * g.C * sizeof(float), 256);
     m.off_edge = o;   o += round_up(tiles * 6 * g.C * sizeof(float), 256);
     m.off_cpart = o;  o += round_up(tiles * g.C * 5 * sizeof(float), 256);
     m.total = o;
@@ -535,19 +536,22 @@ int cawn_phase_accumulate_bwd_dynamic(const cawn_params *params, const void *sav
                       grad_state_in, workspace, workspace_bytes, cuda_stream);
 }
 
-int cawn_mixing_bwd(const cawn_params *params, const float *h, const float *conv_w, const float *conv_bias,
-                    const float *gamma, const float *theta, const void *saved_states, const void *state_in,
-                    const void *grad_y, const void *grad_state_out, float *grad_h, float *grad_conv_w,
-                    float *grad_conv_bias, float *grad_gamma, float *grad_theta, void *grad_state_in,
-                    void *workspace, size_t workspace_bytes, void *cuda_stream)
+// Backward of the fused path, static (gamma) or time-varying (gamma_logit, freq_bias) retention.
+static int mix_bwd_common(const cawn_params *params, bool dyn, const float *h, const float *conv_w, const float *conv_bias,
+                          const float *gamma, const float *gamma_logit, const float *freq_bias,
+                          const float *theta, const void *saved_states, const void *state_in,
+                          const void *grad_y, const void *grad_state_out, float *grad_h, float *grad_conv_w,
+                          float *grad_conv_bias, float *grad_gamma, float *grad_logit, float *grad_fbias,
+                          float *grad_theta, void *grad_state_in,
+                          void *workspace, size_t workspace_bytes, void *cuda_stream)
 {
     int rc = check_params(params);
     if (rc != CAWN_OK) return rc;
     if (params->flags & kBf16Flags) return CAWN_ERR_UNSUPPORTED;   // fp32 storage only here
-    if (params->conv_k < 1 || params->conv_k > 4 || (params->flags & CAWN_FLAG_RETENTION_DYNAMIC))
-        return CAWN_ERR_UNSUPPORTED;
+    if (params->conv_k < 1 || params->conv_k > 4) return CAWN_ERR_UNSUPPORTED;
     if ((params->flags & CAWN_FLAG_PRELUDE_CLAMP_SILU) && params->gate_eps > 0.4f) return CAWN_ERR_UNSUPPORTED;
-    if (conv_w == nullptr || gamma == nullptr || theta == nullptr || workspace == nullptr) return CAWN_ERR_NULL_POINTER;
+    if (conv_w == nullptr || theta == nullptr || workspace == nullptr) return CAWN_ERR_NULL_POINTER;
+    if (dyn ? (gamma_logit == nullptr || freq_bias == nullptr) : gamma == nullptr) return CAWN_ERR_NULL_POINTER;
     if (params->L > 0 && (h == nullptr || grad_y == nullptr || grad_h == nullptr)) return CAWN_ERR_NULL_POINTER;
     if (!aligned(h, 16) || !aligned(grad_h, 16) || !aligned(workspace, 16) || !aligned(state_in, 16) ||
         !aligned(grad_state_out, 16) || !aligned(grad_state_in, 16))
@@ -560,7 +564,7 @@ int cawn_mixing_bwd(const cawn_params *params, const float *h, const float *conv
     cudaStream_t st = (cudaStream_t)cuda_stream;
     const int C = g.C, Kc = params->conv_k, Kh = Kc - 1;
     const size_t tail_off = round_up((size_t)params->B * C * sizeof(float2), 16);
-    const bool want_scan_param = grad_gamma != nullptr || grad_theta != nullptr;
+    const bool want_scan_param = grad_gamma != nullptr || grad_theta != nullptr || grad_logit != nullptr || grad_fbias != nullptr;
     const bool want_conv_param = grad_conv_w != nullptr || grad_conv_bias != nullptr;
     if (params->L > 0 && want_scan_param && saved_states == nullptr) return CAWN_ERR_NULL_POINTER;
     if (!aligned(saved_states, 16) || !aligned(grad_y, 16)) return CAWN_ERR_MISALIGNED;
@@ -577,11 +581,17 @@ int cawn_mixing_bwd(const cawn_params *params, const float *h, const float *conv
         if (grad_conv_bias && cudaMemsetAsync(grad_conv_bias, 0, (size_t)C * sizeof(float), st) != cudaSuccess) return CAWN_ERR_CUDA;
         if (grad_gamma && cudaMemsetAsync(grad_gamma, 0, (size_t)C * sizeof(float), st) != cudaSuccess) return CAWN_ERR_CUDA;
         if (grad_theta && cudaMemsetAsync(grad_theta, 0, (size_t)C * sizeof(float), st) != cudaSuccess) return CAWN_ERR_CUDA;
+        if (grad_fbias && cudaMemsetAsync(grad_fbias, 0, (size_t)params->F * sizeof(float), st) != cudaSuccess) return CAWN_ERR_CUDA;
         return CAWN_OK;
     }
+    // the logit gradient is accumulated with atomic adds: it starts from zero
+    if (grad_logit != nullptr &&
+        cudaMemsetAsync(grad_logit, 0, (size_t)params->B * (size_t)params->L * params->H * sizeof(float), st) != cudaSuccess)
+        return CAWN_ERR_CUDA;
 
     char *base = reinterpret_cast<char *>(workspace);
     float2 *qpart = reinterpret_cast<float2 *>(base + lay.off_qpart);
+    float *spart = reinterpret_cast<float *>(base + lay.off_spart);
     float *edge = reinterpret_cast<float *>(base + lay.off_edge);
     float *cpart = reinterpret_cast<float *>(base + lay.off_cpart);
     const float *tail_in = nullptr, *dtail_out = nullptr;
@@ -608,13 +618,16 @@ int cawn_mixing_bwd(const cawn_params *params, const float *h, const float *conv
     sp.clampv = params->grad_clamp_abs > 0.f ? params->grad_clamp_abs : 0.f;
     sp.poll_limit = kPollLimit;
     sp.H = params->H; sp.F = params->F;
+    sp.gamma_logit = gamma_logit; sp.freq_bias = freq_bias;
+    sp.grad_logit = (dyn && want_scan_param) ? grad_logit : nullptr;
+    sp.spart = (dyn && want_scan_param && grad_fbias != nullptr) ? spart : nullptr;
     sp.hid = h; sp.conv_w = conv_w; sp.conv_bias = conv_bias; sp.tail_in = tail_in;
     sp.conv_k = Kc;
     sp.clamp_silu = (params->flags & CAWN_FLAG_PRELUDE_CLAMP_SILU) ? 1 : 0;
     sp.gate_tau = params->gate_tau;
     sp.edge_du = edge;
     sp.cpart = want_conv_param ? cpart : nullptr;
-    if (launch_mix_bwd(ts, sp, st) != cudaSuccess) return CAWN_ERR_CUDA;
+    if ((dyn ? launch_mix_bwd_dynamic(ts, sp, st) : launch_mix_bwd(ts, sp, st)) != cudaSuccess) return CAWN_ERR_CUDA;
 
     // 2. rows at the tile seams and the gradient of the carried conv history
     {
@@ -627,8 +640,13 @@ int cawn_mixing_bwd(const cawn_params *params, const float *h, const float *conv
     const int warps = 8;
     if (want_scan_param) {
         cawn_bwd_finalize_kernel<<<(C + warps - 1) / warps, warps * 32, 0, st>>>(
-            qpart, params->B * g.K, C, gamma, theta, grad_gamma, grad_theta, sp.clampv);
+            qpart, params->B * g.K, C, dyn ? nullptr : gamma, theta, dyn ? nullptr : grad_gamma, grad_theta, sp.clampv);
         if (cudaGetLastError() != cudaSuccess) return CAWN_ERR_CUDA;
+        if (dyn && grad_fbias != nullptr) {
+            cawn_bwd_freq_bias_kernel<<<(params->F + warps - 1) / warps, warps * 32, 0, st>>>(
+                spart, params->B * g.K, params->H, params->F, grad_fbias);
+            if (cudaGetLastError() != cudaSuccess) return CAWN_ERR_CUDA;
+        }
     }
     if (want_conv_param) {
         cawn_conv_grad_finalize_kernel<<<(C + warps - 1) / warps, warps * 32, 0, st>>>(
@@ -636,6 +654,31 @@ int cawn_mixing_bwd(const cawn_params *params, const float *h, const float *conv
         if (cudaGetLastError() != cudaSuccess) return CAWN_ERR_CUDA;
     }
     return CAWN_OK;
+}
+
+int cawn_mixing_bwd(const cawn_params *params, const float *h, const float *conv_w, const float *conv_bias,
+                    const float *gamma, const float *theta, const void *saved_states, const void *state_in,
+                    const void *grad_y, const void *grad_state_out, float *grad_h, float *grad_conv_w,
+                    float *grad_conv_bias, float *grad_gamma, float *grad_theta, void *grad_state_in,
+                    void *workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    if (params != nullptr && (params->flags & CAWN_FLAG_RETENTION_DYNAMIC)) return CAWN_ERR_UNSUPPORTED;
+    return mix_bwd_common(params, false, h, conv_w, conv_bias, gamma, nullptr, nullptr, theta, saved_states, state_in,
+                          grad_y, grad_state_out, grad_h, grad_conv_w, grad_conv_bias, grad_gamma, nullptr, nullptr,
+                          grad_theta, grad_state_in, workspace, workspace_bytes, cuda_stream);
+}
+
+int cawn_mixing_bwd_dynamic(const cawn_params *params, const float *h, const float *conv_w, const float *conv_bias,
+                            const float *gamma_logit, const float *freq_bias, const float *theta,
+                            const void *saved_states, const void *state_in,
+                            const void *grad_y, const void *grad_state_out, float *grad_h, float *grad_conv_w,
+                            float *grad_conv_bias, float *grad_gamma_logit, float *grad_freq_bias, float *grad_theta,
+                            void *grad_state_in, void *workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    if (params != nullptr && !(params->flags & CAWN_FLAG_RETENTION_DYNAMIC)) return CAWN_ERR_INVALID_ARG;
+    return mix_bwd_common(params, true, h, conv_w, conv_bias, nullptr, gamma_logit, freq_bias, theta, saved_states, state_in,
+                          grad_y, grad_state_out, grad_h, grad_conv_w, grad_conv_bias, nullptr, grad_gamma_logit,
+                          grad_freq_bias, grad_theta, grad_state_in, workspace, workspace_bytes, cuda_stream);
 }
 
 int cawn_state_carry(const cawn_params *params, const void *state_prev, const void *state_local,

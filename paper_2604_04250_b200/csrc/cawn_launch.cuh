@@ -21,5 +21,6 @@ cudaError_t launch_fused_bf16(TileShape ts, const ScanParams &sp, cudaStream_t s
 cudaError_t launch_bwd_static(TileShape ts, const ScanParams &sp, cudaStream_t st);    // reverse scan
 cudaError_t launch_bwd_dynamic(TileShape ts, const ScanParams &sp, cudaStream_t st);
 cudaError_t launch_mix_bwd(TileShape ts, const ScanParams &sp, cudaStream_t st);       // reverse scan + prelude backward
+cudaError_t launch_mix_bwd_dynamic(TileShape ts, const ScanParams &sp, cudaStream_t st);
 
 }  // namespace cawn

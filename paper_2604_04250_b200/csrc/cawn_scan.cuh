@@ -271,7 +271,6 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
     static_assert(!(EAR && (DYN || kind_is_bwd(KIND))), "the Ear epilogue belongs to the static forward");
     static_assert(IO == IO_F32 || (!EAR && !DYN && !kind_is_bwd(KIND)), "bf16 storage is built for the static forward");
     constexpr bool IN16 = (IO & IO_IN_BF16) != 0, OUT16 = (IO & IO_OUT_BF16) != 0;
-    static_assert(!(DYN && KIND == KIND_MIXBWD), "time-varying retention is not built for the fused path");
     constexpr bool REV = kind_is_bwd(KIND);
     constexpr bool MIX = (KIND == KIND_MIXBWD);
     constexpr int TILE = T * W;

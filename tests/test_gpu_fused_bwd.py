@@ -135,3 +135,51 @@ def test_mixing_bwd_config4_shape_sampled():
         ref = reference(sub, cfg.gate_eps)
         assert floored_rel_err(got["dh"][b:b + 1], ref["dh"]) < TOL
         assert floored_rel_err(got["dstate_in"][b:b + 1], ref["dstate_in"]) < TOL
+
+
+@pytest.mark.parametrize("B,L,H,F,Kc", [(1, 1, 1, 64, 4), (2, 70, 2, 64, 4), (1, 200, 3, 32, 3), (2, 131, 5, 16, 4), (1, 300, 3, 11, 4),
+                                        (1, 515, 12, 64, 4), (2, 20, 2, 64, 2)])
+def test_mixing_bwd_with_dynamic_retention(B, L, H, F, Kc):
+    """Backward of the paper's own layer form: conv prelude, gated push, retention per token and head."""
+    import torch
+    from gpu_util import dev, state_blob, split_blob
+    from paper_2604_04250_b200 import binding as cb
+    C = H * F
+    d = make(B, L, C, Kc, seed=1500 + L)
+    d.update(inputs.dynamic_retention_inputs(B, L, H, F, 1501 + L))
+    eps, tau = 0.1, float(inputs.gate_tau(0.1))
+    tail = d["gso_tail"] if Kc > 1 else None
+    ref = oracle.fused_backward(d["h"], d["conv_w"], None, d["theta"], d["G"], eps, tau, bias=d.get("conv_bias"),
+                                tail_in=d.get("tail_in"), state_in=d["P_in"].astype(np.complex128),
+                                dstate_out=d["gso_P"].astype(np.complex128), dtail_out=tail,
+                                gamma_logit=d["gamma_logit"], freq_bias=d["freq_bias"], H=H)
+    prm = cb.make_params(B, L, H, F, gate_eps=eps, gate_tau=tau, conv_k=Kc, flags=cb.CAWN_FLAG_RETENTION_DYNAMIC)
+    t, w, bias = dev(d["theta"]), dev(d["conv_w"]), dev(d.get("conv_bias"))
+    gl, fb = dev(d["gamma_logit"]), dev(d["freq_bias"])
+    s_in, off = state_blob(B, C, Kc, d["P_in"], d.get("tail_in"))
+    y = torch.empty((B, L, C), dtype=torch.complex64, device="cuda")
+    wf = cb.new_workspace(prm, cb.CAWN_OP_FWD)
+    cb.cawn_phase_accumulate_fwd(prm, dev(d["h"]), None, t, y, wf, conv_w=w, conv_bias=bias, gamma_logit=gl, freq_bias=fb,
+                                 state_in=s_in)
+    assert cb.cawn_poll_status(wf) == 0
+    gso, _ = state_blob(B, C, Kc, d["gso_P"], tail)
+    gsi, _ = state_blob(B, C, Kc)
+    ws = cb.new_workspace(prm, cb.CAWN_OP_MIXING_BWD)
+    nan = float("nan")
+    gh = torch.full((B, L, C), nan, device="cuda")
+    gw, gb = torch.full((C, Kc), nan, device="cuda"), torch.full((C,), nan, device="cuda")
+    ggl, gfb, gt = torch.full((B, L, H), nan, device="cuda"), torch.full((F,), nan, device="cuda"), torch.full((C,), nan, device="cuda")
+    cb.cawn_mixing_bwd_dynamic(prm, dev(d["h"]), w, gl, fb, t, dev(d["G"]), gh, ws, conv_bias=bias, saved_states=y, state_in=s_in,
+                               grad_state_out=gso, grad_conv_w=gw, grad_conv_bias=gb, grad_gamma_logit=ggl, grad_freq_bias=gfb,
+                               grad_theta=gt, grad_state_in=gsi)
+    assert cb.cawn_poll_status(ws) == 0
+    dP, dtail = split_blob(gsi, off, B, C, Kc)
+    assert floored_rel_err(gh.cpu().numpy(), ref["dh"]) < TOL
+    assert floored_rel_err(gw.cpu().numpy(), ref["dw"]) < TOL
+    assert floored_rel_err(gb.cpu().numpy(), ref["dbias"]) < TOL
+    assert floored_rel_err(ggl.cpu().numpy(), ref["dgamma_logit"]) < TOL
+    assert floored_rel_err(gfb.cpu().numpy(), ref["dfreq_bias"]) < TOL
+    assert floored_rel_err(gt.cpu().numpy(), ref["dtheta"]) < TOL
+    assert floored_rel_err(dP, ref["dstate_in"]) < TOL
+    if Kc > 1:
+        assert floored_rel_err(dtail, ref["dtail_in"]) < TOL
