@@ -276,8 +276,10 @@ CAWN_API int cawn_mixing_bwd_dynamic(const cawn_params *params,
  * Forward with the front of the Convolutional SwiGLU Ear as the scan's epilogue (Eq. (wave_synth)
  * and Section "Projection to Hidden State: The Convolutional SwiGLU Ear", the depth-wise 1-D
  * convolution across the K harmonics).  Everything up to the clamped state y_t is
- * cawn_phase_accumulate_fwd (Cartesian or fused input, static retention only); instead of
- * storing y the kernel writes
+ * cawn_phase_accumulate_fwd (Cartesian or fused input, static or time-varying retention: with
+ * conv_k >= 1 and CAWN_FLAG_RETENTION_DYNAMIC one kernel takes the hidden states through the
+ * paper's whole Resonance mixing step up to the Ear's convolution); instead of storing y the
+ * kernel writes
  *   Z_t = Concat(Re y_t, Im y_t)  viewed as 2H channels (real heads, then imaginary heads) x K
  *   z_conv[b,t,q,k] = ear_bias[q] + sum_j ear_w[q,j] Z_t[q, k + j - (ear_k-1)/2],  zero outside 0..K-1
  * The paper states neither the tap count nor the padding: taken as ear_k taps (1 or 3; other
@@ -287,13 +289,14 @@ CAWN_API int cawn_mixing_bwd_dynamic(const cawn_params *params,
  * z_conv:  [B, L, 2, H, K] float (device, 16-byte aligned), K = params->F; as many bytes as y.
  * state_out (if given) still receives the unclamped, unconvolved P_{L-1} (and the conv history).
  * Limits: K must divide 64 unless H*K <= 64 (a CTA owns 64 adjacent channels and does not read
- * its neighbours' harmonics); CAWN_FLAG_RETENTION_DYNAMIC -> CAWN_ERR_UNSUPPORTED.
+ * its neighbours' harmonics).
  * Other arguments, ownership, stream order and status reporting as cawn_phase_accumulate_fwd.
  */
 CAWN_API int cawn_phase_accumulate_fwd_ear(const cawn_params *params,
                                            const void *input,
                                            const float *gamma, const float *theta,
                                            const float *conv_w, const float *conv_bias,
+                                           const float *gamma_logit, const float *freq_bias,
                                            const void *state_in,
                                            const float *ear_w, const float *ear_bias, int ear_k,
                                            float *z_conv, void *state_out, uint32_t *gate_mask,

@@ -221,6 +221,14 @@ def _cfg4(args, cb, inputs, dev, IND):
                    max(args.steps // 2, 5), args.warmup)
         assert cb.cawn_poll_status(ws) == 0
         _report("cfg4_fused_dynamic_retention", B * L, B * L * (C * 12 + cfg.H * 4), ms, 1)
+        # ... and with the Ear's convolution across the harmonics as the epilogue: the whole mixing step
+        ew, eb = torch.randn((2 * cfg.H, 3), device="cuda"), torch.randn(2 * cfg.H, device="cuda")
+        zs = [y.view(torch.float32).view(B, L, 2, C) for y in ys]
+        ms = _time(lambda i: cb.cawn_phase_accumulate_fwd_ear(prm_d, hs[i % NS], None, t, ew, 3, zs[i % NS], ws, ear_bias=eb,
+                                                              conv_w=w, gamma_logit=gl, freq_bias=fb),
+                   max(args.steps // 2, 5), args.warmup)
+        assert cb.cawn_poll_status(ws) == 0
+        _report("cfg4_fused_dynamic_retention+ear_conv", B * L, B * L * (C * 12 + cfg.H * 4), ms, 1)
     if "bf16" in args.only or not args.only:
         prm16 = cb.make_params(B, L, cfg.H, cfg.F, gate_eps=cfg.gate_eps, gate_tau=float(inputs.gate_tau(cfg.gate_eps)),
                                conv_k=cfg.conv_k, flags=IND | cb.CAWN_FLAG_INPUT_BF16 | cb.CAWN_FLAG_OUTPUT_BF16)

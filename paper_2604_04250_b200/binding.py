@@ -87,7 +87,7 @@ def lib():
         L.cawn_phase_accumulate_bwd.argtypes = [pp, vp, ctypes.c_int, fp, fp, vp, vp, vp, vp, fp, fp, vp, vp, sz, vp]
         L.cawn_phase_accumulate_bwd_dynamic.argtypes = [pp, vp, ctypes.c_int, fp, fp, fp, vp, vp, vp, vp, fp, fp, fp, vp, vp, sz, vp]
         L.cawn_mixing_bwd.argtypes = [pp, fp, fp, fp, fp, fp, vp, vp, vp, vp, fp, fp, fp, fp, fp, vp, vp, sz, vp]
-        L.cawn_phase_accumulate_fwd_ear.argtypes = [pp, vp, fp, fp, fp, fp, vp, fp, fp, ctypes.c_int, fp, vp, vp, vp, sz, vp]
+        L.cawn_phase_accumulate_fwd_ear.argtypes = [pp, vp, fp, fp, fp, fp, fp, fp, vp, fp, fp, ctypes.c_int, fp, vp, vp, vp, sz, vp]
         L.cawn_mixing_bwd_dynamic.argtypes = [pp, fp, fp, fp, fp, fp, fp, vp, vp, vp, vp, fp, fp, fp, fp, fp, fp, vp, vp, sz, vp]
         L.cawn_state_carry.argtypes = [pp, vp, vp, ctypes.c_int64, fp, fp, vp, vp]
         L.cawn_poll_status.argtypes = [vp, vp]
@@ -163,10 +163,11 @@ def cawn_phase_accumulate_fwd(params, input, gamma, theta, y, workspace, conv_w=
 
 
 def cawn_phase_accumulate_fwd_ear(params, input, gamma, theta, ear_w, ear_k, z_conv, workspace, ear_bias=None,
-                                  conv_w=None, conv_bias=None, state_in=None, state_out=None, gate_mask=None,
-                                  stream=None):
+                                  conv_w=None, conv_bias=None, gamma_logit=None, freq_bias=None, state_in=None,
+                                  state_out=None, gate_mask=None, stream=None):
     _check(lib().cawn_phase_accumulate_fwd_ear(
-        ctypes.byref(params), _dp(input), _dp(gamma), _dp(theta), _dp(conv_w), _dp(conv_bias), _dp(state_in),
+        ctypes.byref(params), _dp(input), _dp(gamma), _dp(theta), _dp(conv_w), _dp(conv_bias), _dp(gamma_logit),
+        _dp(freq_bias), _dp(state_in),
         _dp(ear_w), _dp(ear_bias), int(ear_k), _dp(z_conv), _dp(state_out), _dp(gate_mask),
         _dp(workspace), workspace.numel() * workspace.element_size(), _stream(stream)),
         "cawn_phase_accumulate_fwd_ear")

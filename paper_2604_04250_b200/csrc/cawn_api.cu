@@ -134,12 +134,12 @@ inline int io_of(const cawn_params *p)
 inline cudaError_t launch_fwd(TileShape ts, const ScanParams &sp, cudaStream_t st, bool dyn = false, int io = 0)
 {
     if (io != 0) return launch_fwd_bf16(ts, sp, st, io);
-    if (sp.ear_w != nullptr) return launch_fwd_ear(ts, sp, st);
+    if (sp.ear_w != nullptr) return dyn ? launch_fwd_ear_dynamic(ts, sp, st) : launch_fwd_ear(ts, sp, st);
     return dyn ? launch_fwd_dynamic(ts, sp, st) : launch_fwd_static(ts, sp, st);
 }
 inline cudaError_t launch_fused(TileShape ts, const ScanParams &sp, cudaStream_t st, int io = 0, bool dyn = false)
 {
-    if (dyn) return launch_fused_dynamic(ts, sp, st);
+    if (dyn) return sp.ear_w != nullptr ? launch_fused_ear_dynamic(ts, sp, st) : launch_fused_dynamic(ts, sp, st);
     if (io != 0) return launch_fused_bf16(ts, sp, st, io);
     return sp.ear_w != nullptr ? launch_fused_ear(ts, sp, st) : launch_fused_plain(ts, sp, st);
 }
@@ -296,7 +296,6 @@ static int fwd_common(const cawn_params *params, const void *input,
     if (io != 0 && (dyn || ear_w != nullptr)) return CAWN_ERR_UNSUPPORTED;
     if (ear_w != nullptr) {
         if (ear_k != 1 && ear_k != 3) return CAWN_ERR_UNSUPPORTED;
-        if (dyn) return CAWN_ERR_UNSUPPORTED;
         // a CTA owns 64 adjacent channels: a head's harmonics must not straddle two of them
         if ((long long)params->H * params->F > 64 && 64 % params->F != 0) return CAWN_ERR_UNSUPPORTED;
         if (!aligned(ear_w, 4) || !aligned(ear_bias, 4)) return CAWN_ERR_MISALIGNED;
@@ -388,13 +387,14 @@ int cawn_phase_accumulate_fwd(const cawn_params *params, const void *input,
 int cawn_phase_accumulate_fwd_ear(const cawn_params *params, const void *input,
                                   const float *gamma, const float *theta,
                                   const float *conv_w, const float *conv_bias,
+                                  const float *gamma_logit, const float *freq_bias,
                                   const void *state_in,
                                   const float *ear_w, const float *ear_bias, int ear_k,
                                   float *z_conv, void *state_out, uint32_t *gate_mask,
                                   void *workspace, size_t workspace_bytes, void *cuda_stream)
 {
     if (ear_w == nullptr) return CAWN_ERR_NULL_POINTER;
-    return fwd_common(params, input, gamma, theta, conv_w, conv_bias, nullptr, nullptr, state_in, z_conv,
+    return fwd_common(params, input, gamma, theta, conv_w, conv_bias, gamma_logit, freq_bias, state_in, z_conv,
                       state_out, gate_mask, workspace, workspace_bytes, cuda_stream, ear_w, ear_bias, ear_k);
 }
 

@@ -14,6 +14,8 @@ cudaError_t launch_fwd_dynamic(TileShape ts, const ScanParams &sp, cudaStream_t 
 cudaError_t launch_fwd_ear(TileShape ts, const ScanParams &sp, cudaStream_t st);       // Ear epilogue
 cudaError_t launch_fused_plain(TileShape ts, const ScanParams &sp, cudaStream_t st);   // fused mixing path
 cudaError_t launch_fused_ear(TileShape ts, const ScanParams &sp, cudaStream_t st);
+cudaError_t launch_fwd_ear_dynamic(TileShape ts, const ScanParams &sp, cudaStream_t st);   // Ear epilogue + time-varying retention
+cudaError_t launch_fused_ear_dynamic(TileShape ts, const ScanParams &sp, cudaStream_t st);
 cudaError_t launch_fused_dynamic(TileShape ts, const ScanParams &sp, cudaStream_t st); // fused path, time-varying retention
 // bf16 storage of the input (io & IO_IN_BF16) and / or the output (io & IO_OUT_BF16); io != 0
 cudaError_t launch_fwd_bf16(TileShape ts, const ScanParams &sp, cudaStream_t st, int io);

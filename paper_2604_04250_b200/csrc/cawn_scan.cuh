@@ -268,7 +268,7 @@ template <int T, int W, int KIND, bool VEC, bool DYN, bool FULL, bool EAR = fals
 __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, KIND, DYN> &sm,
                                           const int g, const int b, const int k)
 {
-    static_assert(!(EAR && (DYN || kind_is_bwd(KIND))), "the Ear epilogue belongs to the static forward");
+    static_assert(!(EAR && kind_is_bwd(KIND)), "the Ear epilogue belongs to the forward");
     static_assert(IO == IO_F32 || (!EAR && !DYN && !kind_is_bwd(KIND)), "bf16 storage is built for the static forward");
     constexpr bool IN16 = (IO & IO_IN_BF16) != 0, OUT16 = (IO & IO_OUT_BF16) != 0;
     constexpr bool REV = kind_is_bwd(KIND);

@@ -125,3 +125,42 @@ def test_ear_refusals():
     with pytest.raises(cb.CawnError) as e:
         cb.cawn_phase_accumulate_fwd_ear(prm, x, g, g, one, 5, z, ws)
     assert e.value.status == cb.CAWN_ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("B,L,H,F,fused", [(2, 200, 2, 64, True), (1, 333, 3, 32, True), (1, 515, 12, 64, True),
+                                            (2, 150, 4, 16, False), (1, 20, 1, 64, True)])
+def test_ear_with_dynamic_retention(B, L, H, F, fused):
+    """The whole Resonance mixing step in one kernel: (conv prelude, gated push,) recurrence with
+    per-token retention, clamp, Ear convolution across the harmonics."""
+    import torch
+    from gpu_util import dev, state_blob
+    from paper_2604_04250_b200 import binding as cb
+    C = H * F
+    eps, clamp = 0.1, 3.0
+    ew, eb = ear_taps(H, 3, 810 + L)
+    dd = inputs.dynamic_retention_inputs(B, L, H, F, 811 + L)
+    gl, fb = dev(dd["gamma_logit"]), dev(dd["freq_bias"])
+    z = torch.full((B, L, 2, H, F), float("nan"), device="cuda")
+    kw = dict(gamma_logit=dd["gamma_logit"], freq_bias=dd["freq_bias"], H=H)
+    if fused:
+        Kc = 4
+        d = inputs.fused_inputs(B, L, C, 812 + L, conv_k=Kc, with_tail=True)
+        tau = float(inputs.gate_tau(eps))
+        prm = cb.make_params(B, L, H, F, gate_eps=eps, gate_tau=tau, clamp_abs=clamp, conv_k=Kc, flags=cb.CAWN_FLAG_RETENTION_DYNAMIC)
+        s_in, _ = state_blob(B, C, Kc, None, d["tail_in"])
+        ws = cb.new_workspace(prm, cb.CAWN_OP_FWD)
+        cb.cawn_phase_accumulate_fwd_ear(prm, dev(d["h"]), None, dev(d["theta"]), dev(ew), 3, z, ws, ear_bias=dev(eb),
+                                         conv_w=dev(d["conv_w"]), conv_bias=dev(d.get("conv_bias")), gamma_logit=gl,
+                                         freq_bias=fb, state_in=s_in)
+        y, _, _, _ = oracle.fused_forward(d["h"], d["conv_w"], None, d["theta"], eps, tau, bias=d.get("conv_bias"),
+                                          tail_in=d["tail_in"], clamp_abs=clamp, **kw)
+    else:
+        d = inputs.scan_inputs(B, L, C, 813 + L)
+        prm = cb.make_params(B, L, H, F, gate_eps=eps, clamp_abs=clamp, flags=cb.CAWN_FLAG_RETENTION_DYNAMIC)
+        ws = cb.new_workspace(prm, cb.CAWN_OP_FWD)
+        cb.cawn_phase_accumulate_fwd_ear(prm, dev(d["p"]), None, dev(d["theta"]), dev(ew), 3, z, ws, ear_bias=dev(eb),
+                                         gamma_logit=gl, freq_bias=fb)
+        zz, _ = oracle.gate(d["p"], eps)
+        y, _ = oracle.scan(zz, d["theta"], clamp_abs=clamp, **kw)
+    assert cb.cawn_poll_status(ws) == 0
+    assert floored_rel_err(z.cpu().numpy(), oracle.ear_conv(y, ew, eb, H, F)) < TOL
