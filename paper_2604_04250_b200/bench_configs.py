@@ -104,8 +104,10 @@ def main():
         dd = inputs.dynamic_retention_inputs(B, L, cfg.H, cfg.F, 7)
         gl, fb = dev(dd["gamma_logit"]), dev(dd["freq_bias"])
         prm_d = cb.make_params(B, L, cfg.H, cfg.F, gate_eps=cfg.gate_eps, flags=IND | cb.CAWN_FLAG_RETENTION_DYNAMIC)
-        ms = _time(lambda i: cb.cawn_phase_accumulate_fwd(prm_d, ps[i % NS], None, t, ys[i % NS], ws, gamma_logit=gl, freq_bias=fb),
+        ws_d = cb.new_workspace(prm_d, cb.CAWN_OP_FWD)
+        ms = _time(lambda i: cb.cawn_phase_accumulate_fwd(prm_d, ps[i % NS], None, t, ys[i % NS], ws_d, gamma_logit=gl, freq_bias=fb),
                    args.steps, args.warmup)
+        assert cb.cawn_poll_status(ws_d) == 0
         _report("cfg1_train_fwd_dynamic_retention", B * L, B * L * (C * 16 + cfg.H * 4), ms, 1)
     assert cb.cawn_poll_status(ws) == 0
     del ps, ys, masks
