@@ -434,26 +434,30 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
     }
 
     // ---- per-channel coefficients, in double, rounded once --------------------------------
-    // Three independent tasks per channel, one thread each: a^n = gamma^n (cos n theta, sin n theta)
-    // for n = 1, T, TILE.  n theta is exact in double (theta is a float, n a small integer).
-    for (int idx = tid; idx < 192; idx += W * 32) {
-        const int task = idx >> 6, cl = idx & 63, ch = g * 64 + cl;
-        float re = 0.f, im = 0.f;
+    // One thread per channel: a = gamma (cos theta, sin theta) from one sincos, then a^T and
+    // a^TILE = (a^T)^W by square-and-multiply, all in double (a dozen complex products, each good to
+    // 2^-52), each rounded to fp32 once.
+    for (int cl = tid; cl < 64; cl += W * 32) {
+        const int ch = g * 64 + cl;
+        double c1r = 0.0, c1i = 0.0, cTr = 0.0, cTi = 0.0, cAr = 0.0, cAi = 0.0;
         if (ch < C) {
-            const int n = task == 0 ? 1 : (task == 1 ? T : TILE);
-            const double gm = DYN ? 1.0 : (double)prm.gamma[ch], th = (double)prm.theta[ch];
-            double mag = 1.0, base = gm;
-            for (int m = n; m > 0; m >>= 1) {            // gamma^n by square-and-multiply
-                if (m & 1) mag *= base;
-                base *= base;
-            }
+            const double gm = DYN ? 1.0 : (double)prm.gamma[ch];
             double sn, cs;
-            sincos(th * (double)n, &sn, &cs);
-            re = (float)(mag * cs);
-            im = (float)(REV ? -(mag * sn) : mag * sn);
+            sincos((double)prm.theta[ch], &sn, &cs);
+            c1r = gm * cs;
+            c1i = REV ? -(gm * sn) : gm * sn;
+            auto cpow = [](double br, double bi, int n, double &rr, double &ri) {
+                rr = 1.0; ri = 0.0;
+                for (int m = n; m > 0; m >>= 1) {
+                    if (m & 1) { const double t = rr * br - ri * bi; ri = rr * bi + ri * br; rr = t; }
+                    const double t = br * br - bi * bi; bi = 2.0 * br * bi; br = t;
+                }
+            };
+            cpow(c1r, c1i, T, cTr, cTi);
+            cpow(cTr, cTi, W, cAr, cAi);
         }
-        sm.sCoef[cl][2 * task] = re;
-        sm.sCoef[cl][2 * task + 1] = im;
+        float *o = sm.sCoef[cl];
+        o[0] = (float)c1r; o[1] = (float)c1i; o[2] = (float)cTr; o[3] = (float)cTi; o[4] = (float)cAr; o[5] = (float)cAi;
     }
     // everything below touches what the previous launch may have written (workspace, states)
     if (early && KIND != KIND_FUSED) grid_wait_previous();
