@@ -943,7 +943,10 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
                     if (vB) { __stcs(zr + 1, zrB); __stcs(zi + 1, ziB); }
                 }
             } else if (VEC) {
-                if (vA) __stcs(reinterpret_cast<float4 *>(r), o);
+                // 16-byte rows go out as st.global.cg (kept in L2 until evicted: measured 0.5 us faster on
+                // the training shape than the evict-first form, which stays the better one for the
+                // narrower stores of the other output forms)
+                if (vA) __stcg(reinterpret_cast<float4 *>(r), o);
             } else {
                 float2 *r2 = reinterpret_cast<float2 *>(r);
                 if (vA) __stcs(r2, make_float2(o.x, o.y));
