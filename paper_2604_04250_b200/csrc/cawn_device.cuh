@@ -86,7 +86,8 @@ __device__ __forceinline__ uint4 ld_record(const uint4 *p)
 // epoch and hook of a workspace header in one access
 __device__ __forceinline__ void ld_epoch_hook(const void *hdr, unsigned long long &epoch, unsigned &hook)
 {
-    unsigned x, y, z, w;
+    unsigned x, y, z;
+    [[maybe_unused]] unsigned w;                         // the arrival count: not used here
     asm volatile("ld.volatile.global.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(x), "=r"(y), "=r"(z), "=r"(w) : "l"(hdr) : "memory");
     epoch = ((unsigned long long)y << 32) | x;
     hook = z;

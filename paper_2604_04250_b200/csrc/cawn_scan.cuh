@@ -229,7 +229,9 @@ __device__ __forceinline__ void fetch_rows(float4 *dst, uint32_t dst_s, const ch
     if constexpr (I < T) {
         const bool row = valid(I);
         fetch_piece<VEC, I * 512, HALF>(dst, dst_s, row_ptr(src, step, I), row && vA, row && vB);
-        if constexpr (GR > 0 && (I + 1) % GR == 0) cp_async_commit();
+        if constexpr (GR > 0) {
+            if constexpr ((I + 1) % GR == 0) cp_async_commit();
+        }
         fetch_rows<VEC, T, GR, I + 1, HALF>(dst, dst_s, src, step, vA, vB, valid);
     }
 }
