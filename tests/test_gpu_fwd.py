@@ -167,7 +167,7 @@ def test_host_buffer_entry_point():
     assert np.array_equal(unpack_mask(m.numpy().view(np.uint32), C), m_ref)
 
 
-@pytest.mark.parametrize("B,L,C", [(4, 4096, 128), (11, 2048, 64), (1, 20000, 128), (1, 9000, 192)])
+@pytest.mark.parametrize("B,L,C", [(4, 4096, 128), (11, 2048, 64), (1, 20000, 128), (1, 9000, 192), (2, 16500, 128), (8, 4100, 256)])
 def test_host_buffer_entry_point_sliced(B, L, C):
     """Calls of 8 MB and more go through the two copy streams in slices: batch rows for B >= 2,
     stretches of time with the state carried for B = 1.  Two calls in a row reuse the pipes."""
