@@ -315,21 +315,47 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
     }
     const bool early = !REV && prm.early_loads != 0;
     if (!early) grid_wait_previous();
-    // Fused path: the hidden rows (floats) are staged in the upper part of the tile, behind
-    // kHalo rows of history; phase 1 takes them into registers before the pushes overwrite them.
-    float *const hs = reinterpret_cast<float *>(&sm.tile[0][0][0]) + (TILE * 128 - (TILE + kHalo) * 64);
+    // Fused path: every warp stages its own T hidden rows (floats) behind kHalo rows of history in
+    // the upper part of its own T x 512-byte slice of the tile, row r at byte 256 (T - 3) + 256 r
+    // (r < kHalo: history).  The pushes the warp later writes into the same slice (row i at byte
+    // 512 i) reach hidden row r only at step i >= (r + 12) / 2: the rows are read a copy group (GR)
+    // at a time, rows i+3 .. i+GR+2 at step i = 0, GR, ..., and (r + 12) / 2 >= the step whose group
+    // holds r; the warp synchronises between reading a group and writing its pushes.
+    // No other warp touches the slice, so a warp starts as soon as its own first rows have landed.
+    static_assert(KIND != KIND_FUSED || T == 16 || T == 4, "slice layout of the fused path is checked for 16 and 4 rows");
+    float *const hstage = reinterpret_cast<float *>(&sm.tile[0][w * T][0]) + (T * 128 - (T + kHalo) * 64) + 2 * lane;
+    bool fused_tail_group = false;                      // this thread committed one more group (carried history)
     if constexpr (KIND == KIND_FUSED) {
         const float *hin = reinterpret_cast<const float *>(prm.in);
         const unsigned short *hin16 = reinterpret_cast<const unsigned short *>(prm.in);
-        float *mine = hs + (kHalo + w * T) * 64 + 2 * lane;
+        const int Kh = prm.conv_k - 1;
+        // a bf16 hidden value of a history row is kept as the float it widens to
+        auto widen = [](unsigned short v) -> float { return __uint_as_float((unsigned)v << 16); };
+        // history rows that are earlier rows of h (they travel with the first group of own rows)
+#pragma unroll
+        for (int j = 0; j < kHalo; ++j) {
+            const long long t = s0 - kHalo + j;
+            float *d = hstage + j * 64;
+            if (j >= kHalo - Kh && t >= 0 && t < L) {
+                if constexpr (IN16) {
+                    const unsigned short *s16 = hin16 + ((long long)b * L + t) * C + c0;
+                    d[0] = vA ? widen(s16[0]) : 0.f;
+                    d[1] = vB ? widen(s16[1]) : 0.f;
+                } else {
+                    const float *src = hin + ((long long)b * L + t) * C + c0;
+                    if (vA) cp_async4(smem_addr(d), src); else d[0] = 0.f;
+                    if (vB) cp_async4(smem_addr(d + 1), src + 1); else d[1] = 0.f;
+                }
+            } else if (t >= 0 || prm.tail_in == nullptr || j < kHalo - Kh) {
+                d[0] = 0.f; d[1] = 0.f;                 // no such tap, or no carried history
+            }
+        }
         const float *r = hin + e0;
         const unsigned short *r16 = hin16 + e0;
-        // a bf16 hidden value is kept in its float slot as the float it widens to
-        auto widen = [](unsigned short v) -> float { return __uint_as_float((unsigned)v << 16); };
 #pragma unroll
         for (int i = 0; i < T; ++i) {
             const bool row = FULL || i < nvalid;
-            float *d = mine + i * 64;
+            float *d = hstage + (kHalo + i) * 64;
             if constexpr (IN16) {
                 // the pair of bf16 goes into the first word of the slot; phase 1 widens it
                 if (VEC) {
@@ -348,37 +374,25 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
                 if (row && vB) cp_async4(smem_addr(d + 1), r + 1); else d[1] = 0.f;
             }
             r += C;
+            if ((i + 1) % GR == 0) cp_async_commit();
         }
-        // history rows in front of the tile: earlier rows of h, or the carried tail before t = 0
-        // (the tail is the previous call's output: never before that call is complete)
-        const int Kh = prm.conv_k - 1;
+        // history rows before t = 0 come from the carried tail: the previous call's output, never
+        // read before that call is complete
         if (early) grid_wait_previous();
-        if (w == 0) {
-            const long long t0 = (long long)k * TILE;
+        if (s0 < kHalo && prm.tail_in != nullptr) {
 #pragma unroll
             for (int j = 0; j < kHalo; ++j) {
-                const long long t = t0 - kHalo + j;
-                float *d = hs + j * 64 + 2 * lane;
-                const float *src = nullptr;
-                if (j >= kHalo - Kh) {
-                    if (t >= 0) src = hin + ((long long)b * L + t) * C + c0;
-                    else if (prm.tail_in != nullptr) src = prm.tail_in + ((long long)b * Kh + (Kh + t)) * C + c0;
+                const long long t = s0 - kHalo + j;
+                if (j >= kHalo - Kh && t < 0) {
+                    float *d = hstage + j * 64;
+                    const float *src = prm.tail_in + ((long long)b * Kh + (Kh + t)) * C + c0;
+                    if (vA) cp_async4(smem_addr(d), src); else d[0] = 0.f;
+                    if (vB) cp_async4(smem_addr(d + 1), src + 1); else d[1] = 0.f;
                 }
-                if constexpr (IN16) {
-                    // earlier rows of h are bf16 (widened here, stored as floats like the carried
-                    // tail, which is fp32 in the state blob)
-                    if (j >= kHalo - Kh && t >= 0) {
-                        const unsigned short *s16 = hin16 + ((long long)b * L + t) * C + c0;
-                        d[0] = vA ? widen(s16[0]) : 0.f;
-                        d[1] = vB ? widen(s16[1]) : 0.f;
-                        continue;
-                    }
-                }
-                if (src != nullptr && vA) cp_async4(smem_addr(d), src); else d[0] = 0.f;
-                if (src != nullptr && vB) cp_async4(smem_addr(d + 1), src + 1); else d[1] = 0.f;
             }
+            cp_async_commit();
+            fused_tail_group = true;
         }
-        cp_async_commit();
     } else {
         if constexpr (IN16)
             fetch_rows<VEC, T, GR, 0, true>(xs, smem_addr(xs), reinterpret_cast<const char *>(prm.in) + e0 * 4, rowbytes / 2,
@@ -474,7 +488,6 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
         // counted only once the epoch has been read (the increment depends on its value)
         arrived = atomicAdd(&prm.ws->done, 1u + (unsigned)(epoch0 >> 63));
     }
-    if constexpr (KIND == KIND_FUSED) cp_async_wait_all();   // rows are read across threads below
     __syncthreads();                                                           // barrier 1
     float4 a, aT;
     {
@@ -551,21 +564,21 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
         // Temporal Syntax Cache prelude: causal depthwise conv over time (taps right-aligned on
         // the current token, fmaf chain in tap order from the bias), optional clamp + SiLU,
         // magnitude sigmoid(x), phase pi*tanh(x), gate on the conv output, push m (cos, sin).
-        float2 hv[T + kHalo];
-#pragma unroll
-        for (int r = 0; r < T + kHalo; ++r) {
-            const float *slot = hs + (w * T + r) * 64 + 2 * lane;
-            // own rows of a bf16 input are still packed pairs; history rows (r < kHalo as seen
-            // from warp 0, other warps' rows otherwise) follow the same rule row by row
-            if (IN16 && (w * T + r) >= kHalo) hv[r] = bf16x2_to_float2(*reinterpret_cast<const unsigned *>(slot));
-            else hv[r] = *reinterpret_cast<const float2 *>(slot);
-        }
+        // hidden row r of this lane's channel pair (history rows are floats; own rows of a bf16
+        // input are still packed pairs)
+        auto hidden_row = [&](int r) -> float2 {
+            const float *slot = hstage + r * 64;
+            if (IN16 && r >= kHalo) return bf16x2_to_float2(*reinterpret_cast<const unsigned *>(slot));
+            return *reinterpret_cast<const float2 *>(slot);
+        };
         if (early_ptr != nullptr) {
             er0 = ld_record(early_ptr + 2 * lane);
             er1 = ld_record(early_ptr + 2 * lane + 1);
         }
         const int Kc = prm.conv_k;
-        __syncthreads();                 // every thread holds its hidden rows: the staging area may go
+        // the first group of rows (and the history) has landed: the rolling window of the conv
+        if (fused_tail_group) cp_async_wait_all(); else cp_async_wait_pending(NG - 1);
+        float2 hv0 = hidden_row(0), hv1 = hidden_row(1), hv2 = hidden_row(2), hv3, hq[GR];
         const bool act = prm.clamp_silu != 0;
         const float tau = prm.gate_tau;
         const bool want_mask = prm.mask != nullptr;
@@ -597,10 +610,21 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
         }
 #pragma unroll
         for (int i = 0; i < T; ++i) {
-            float2 u = b2;
+            if (i % GR == 0) {
+                // the group's GR new hidden rows come out of the slice together, then the warp
+                // synchronises once: the pushes of these GR steps only reach rows read by now
+                if (i > 0 && !fused_tail_group) cp_async_wait_pending(NG - 1 - i / GR);
 #pragma unroll
-            for (int j = 0; j < 4; ++j)
-                if (j >= 4 - Kc) u = __ffma2_rn(w2[j], hv[i + j], u);     // fmaf per channel, tap order
+                for (int q = 0; q < GR; ++q) hq[q] = hidden_row(i + kHalo + q);
+                __syncwarp();
+            }
+            hv3 = hq[i % GR];
+            float2 u = b2;
+            if (0 >= 4 - Kc) u = __ffma2_rn(w2[0], hv0, u);               // fmaf per channel, tap order
+            if (1 >= 4 - Kc) u = __ffma2_rn(w2[1], hv1, u);
+            if (2 >= 4 - Kc) u = __ffma2_rn(w2[2], hv2, u);
+            u = __ffma2_rn(w2[3], hv3, u);
+            hv0 = hv1; hv1 = hv2; hv2 = hv3;
             float2 x = u;
             if (act) {
                 x.x = fminf(fmaxf(x.x, -50.f), 50.f); x.y = fminf(fmaxf(x.y, -50.f), 50.f);
