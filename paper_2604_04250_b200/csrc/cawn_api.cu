@@ -101,7 +101,7 @@ inline bool grid_ok(const cawn_params *p, const Geometry &g)
 
 // First-wave stagger of the static forward scan: about two thirds of the time one SM's share of
 // HBM bandwidth needs for a tile's input and output.  Device numbers are read once per device.
-void set_stagger(ScanParams &sp, TileShape ts)
+void set_stagger(ScanParams &sp, TileShape ts, int bytes_per_element = 16)
 {
     static int sms[64] = {}, cycles_per_byte_q20[64] = {};
     int dev = 0;
@@ -119,7 +119,7 @@ void set_stagger(ScanParams &sp, TileShape ts)
         cycles_per_byte_q20[dev] = (int)((double)sm_khz * 1e3 / bytes_per_s * 1048576.0);
         sms[dev] = n;
     }
-    const long long tile_bytes = (long long)ts.T * ts.W * 64 * 16;     // input + output of one tile
+    const long long tile_bytes = (long long)ts.T * ts.W * 64 * bytes_per_element;   // input + output of one tile
     sp.stagger_cycles = (int)((tile_bytes * cycles_per_byte_q20[dev] * 2 / 3) >> 20);
     sp.stagger_group = sms[dev];
     sp.stagger_slots = 3;
@@ -367,7 +367,7 @@ static int fwd_common(const cawn_params *params, const void *input,
     }
     sp.gamma_logit = gamma_logit; sp.freq_bias = freq_bias; sp.H = params->H; sp.F = params->F;
     sp.early_loads = (params->flags & CAWN_FLAG_INPUT_INDEPENDENT) ? 1 : 0;
-    if (!dyn && ts.T == 16 && io == 0) set_stagger(sp, ts);
+    if (!dyn && ts.T == 16) set_stagger(sp, ts, ((io & IO_IN_BF16) ? 4 : 8) + ((io & IO_OUT_BF16) ? 4 : 8));
     if (launch_fwd(ts, sp, st, dyn, io) != cudaSuccess) return CAWN_ERR_CUDA;
     return CAWN_OK;
 }
