@@ -46,6 +46,8 @@ cudaError_t launch_scan(const ScanParams &sp, cudaStream_t st)
 template <int KIND, int IO>
 cudaError_t launch_scan_io(TileShape ts, const ScanParams &sp, cudaStream_t st)
 {
+    // (the Cartesian long-call shape exists with and without the gate-mask output compiled in)
+    if (KIND == KIND_FWD && ts.T == 16 && sp.mask == nullptr) return launch_scan<16, 8, KIND, 3, false, false, IO, false>(sp, st);
     if (ts.T == 16) return launch_scan<16, 8, KIND, 3, false, false, IO>(sp, st);
     return launch_scan<4, 4, KIND, 8, false, false, IO>(sp, st);
 }
