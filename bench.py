@@ -32,7 +32,7 @@ BYTES_PER_ELEMENT = 16         # algorithmic: read one complex64 push, write one
 # workload, from the ncu capture summarised in profiles/cawn_scan_fwd_cfg1_ncu.md: 101.4 MB read
 # + 47.4 MB written while an isolated launch runs (the rest of its 100.7 MB of output is still
 # dirty in L2 when it ends).  Set to None whenever the kernel changes after the capture.
-NCU_DRAM_BYTES_PER_LAUNCH = 151179008
+NCU_DRAM_BYTES_PER_LAUNCH = 151096576
 
 
 def workload():
