@@ -55,7 +55,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
         if failed:
             raise RuntimeError("nvcc failed on: " + ", ".join(failed))
         tmp = LIB + ".tmp" + tag
-        subprocess.check_call([nvcc] + NVCC_FLAGS + LINK_FLAGS + ["-o", tmp] + objs)
+        objs.append(tmp)                    # removed below if the link fails half-way
+        subprocess.check_call([nvcc] + NVCC_FLAGS + LINK_FLAGS + ["-o", tmp] + objs[:-1])
         os.replace(tmp, LIB)
     finally:
         for obj in objs:
