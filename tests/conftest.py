@@ -25,3 +25,11 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(scope="session", autouse=True)
+def built_libraries():
+    """Build libcawn.so (nvcc, sm_100a) and the C oracle (gcc) once per session if they are missing or
+    older than their sources; a no-op when they are up to date."""
+    import __graft_entry__ as entry
+    entry.build()
