@@ -177,7 +177,14 @@ def run_ours(args):
     torch.cuda.set_device(local)
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-    cb.lib()                                   # fails loudly if the CUDA library is missing
+    # a fresh checkout has no built library yet: the first local rank builds it (a no-op when it is
+    # up to date), the others wait for it
+    if local == 0:
+        from paper_2604_04250_b200 import build as cuda_build
+        cuda_build.build()
+    if world > 1:
+        dist.barrier()
+    cb.lib()                                   # fails loudly if the CUDA library is still missing
 
     cfg = workload()
     B, L, C = cfg.B, cfg.L, cfg.C
