@@ -3,8 +3,12 @@
  *
  * C ABI.  Every pointer is caller-owned; "device" pointers are CUDA global memory of the
  * current device, "host" pointers are ordinary (preferably pinned) host memory.  The
- * library allocates no memory and keeps no state of its own: scratch lives in a
- * caller-provided workspace.  Calls are asynchronous on the given CUDA stream
+ * library calls no allocator, and its scratch lives in a caller-provided workspace, with two
+ * exceptions that keep state inside the library: cawn_phase_accumulate_fwd_host creates, on its
+ * first large call per device, two copy streams and a handful of events that it keeps and
+ * serialises behind a lock; cawn_phase_accumulate_fwd_static uses a 4 MiB __device__ array that
+ * is part of the library image and shared by all calls on a device (serialise them).
+ * Calls are asynchronous on the given CUDA stream
  * (a cudaStream_t passed as void*; NULL = the legacy default stream) unless stated.
  *
  * Shapes.  B batch, L time steps, H heads, F harmonics per head, C = H*F complex channels,
@@ -372,9 +376,13 @@ CAWN_API int cawn_phase_accumulate_fwd_host(const cawn_params *params,
  *
  * Same operation and arguments as the Cartesian, static-retention cawn_phase_accumulate_fwd
  * (conv_k == 0, no CAWN_FLAG_RETENTION_DYNAMIC), without the workspace pair.
+ * Anything else (conv_k != 0, CAWN_FLAG_RETENTION_DYNAMIC) is refused with CAWN_ERR_UNSUPPORTED;
+ * all arguments are validated before anything is put on the stream.
  * device_status: device pointer to one uint32 or NULL.  When given, the device-side status of
- *               this call (0 or CAWN_ERR_CARRY_TIMEOUT) is copied there on the stream after the
- *               kernel; there is no separate poll call for the built-in scratch.
+ *               this call is copied there on the stream after the kernel: 0, or the bits
+ *               CAWN_ERR_CARRY_TIMEOUT (1) and CAWN_STATUS_NONFINITE (2) or-ed together, as
+ *               cawn_poll_status would return them; there is no separate poll call for the
+ *               built-in scratch.
  *
  * Limits and rules.
  *  - The call is rejected with CAWN_ERR_STATIC_TOO_LARGE, before anything is launched, when

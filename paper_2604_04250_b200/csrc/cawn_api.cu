@@ -26,6 +26,7 @@ inline TileShape bwd_shape(int64_t L) { return L > 32 ? TileShape{8, 8} : TileSh
 // (KP checkpoint slots per chain); MW mask words per row.  Records are 16 bytes per channel.
 struct Geometry {
     int C, G, K, KP, MW;
+    bool fits;                   // the tile count fits a grid dimension (K is clamped when it does not)
     size_t agg_bytes, pre_bytes, rec_bytes;
 };
 inline Geometry geometry(const cawn_params *p, TileShape ts)
@@ -34,8 +35,10 @@ inline Geometry geometry(const cawn_params *p, TileShape ts)
     g.C = p->H * p->F;
     g.G = (g.C + 63) / 64;
     const int64_t tile = (int64_t)ts.T * ts.W;
-    g.K = (int)((p->L + tile - 1) / tile);
-    if (g.K < 1) g.K = 1;
+    int64_t K64 = p->L / tile + (p->L % tile != 0 ? 1 : 0);     // no overflow for any L >= 0
+    if (K64 < 1) K64 = 1;
+    g.fits = K64 <= 65535;
+    g.K = g.fits ? (int)K64 : 65535;
     g.KP = g.K / kWindow + 1;
     g.MW = (g.C + 31) / 32;
     g.agg_bytes = (size_t)p->B * g.G * g.K * 64 * sizeof(uint4);
@@ -82,6 +85,8 @@ int check_params(const cawn_params *p)
                                  CAWN_FLAG_INPUT_BF16 | CAWN_FLAG_OUTPUT_BF16))
         return CAWN_ERR_INVALID_ARG;
     if (!(p->gate_eps >= 0.f)) return CAWN_ERR_INVALID_ARG;
+    // every byte count derived from B*L*C (16 bytes per element at most, a few arrays) must fit 63 bits
+    if ((double)p->B * (double)p->L * (double)p->H * (double)p->F > 1.0e17) return CAWN_ERR_UNSUPPORTED;
     return CAWN_OK;
 }
 
@@ -96,7 +101,7 @@ size_t state_blob_bytes(const cawn_params *p)
 // Grid size check: tiles are a (G, B, K) grid.
 inline bool grid_ok(const cawn_params *p, const Geometry &g)
 {
-    return p->B <= 65535 && g.K <= 65535 && (double)p->B * g.G * g.K < 4294967295.0;
+    return g.fits && p->B <= 65535 && g.K <= 65535 && (double)p->B * g.G * g.K < 4294967295.0;
 }
 
 // First-wave stagger of the static forward scan: about two thirds of the time one SM's share of
@@ -286,7 +291,8 @@ static int fwd_common(const cawn_params *params, const void *input,
                       const float *gamma_logit, const float *freq_bias,
                       const void *state_in, void *y, void *state_out,
                       uint32_t *gate_mask, void *workspace, size_t workspace_bytes,
-                      void *cuda_stream, const float *ear_w, const float *ear_bias, int ear_k)
+                      void *cuda_stream, const float *ear_w, const float *ear_bias, int ear_k,
+                      bool validate_only = false)
 {
     int rc = check_params(params);
     if (rc != CAWN_OK) return rc;
@@ -322,6 +328,7 @@ static int fwd_common(const cawn_params *params, const void *input,
     const Geometry g = geometry(params, ts);
     if (!grid_ok(params, g)) return CAWN_ERR_UNSUPPORTED;
     if (workspace_bytes < sizeof(WsHeader) + g.rec_bytes) return CAWN_ERR_WORKSPACE_TOO_SMALL;
+    if (validate_only) return CAWN_OK;
     cudaStream_t st = (cudaStream_t)cuda_stream;
 
     if (params->L == 0) {               // nothing to scan: the state (and conv history) passes through
@@ -884,11 +891,18 @@ int cawn_phase_accumulate_fwd_static(const cawn_params *params, const void *inpu
     size_t need = 0;
     int rc = cawn_workspace_bytes(params, CAWN_OP_FWD, &need);
     if (rc != CAWN_OK) return rc;
+    if (params->conv_k != 0 || (params->flags & CAWN_FLAG_RETENTION_DYNAMIC)) return CAWN_ERR_UNSUPPORTED;
     if (need > (size_t)CAWN_STATIC_SCRATCH_BYTES) return CAWN_ERR_STATIC_TOO_LARGE;
     if (!aligned(device_status, 4)) return CAWN_ERR_MISALIGNED;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    // every argument is checked before anything is put on the stream (the workspace pointer of this
+    // dry run only has to be non-NULL and aligned: nothing dereferences it)
+    rc = fwd_common(params, input, gamma, theta, nullptr, nullptr, nullptr, nullptr, state_in, y, state_out, gate_mask,
+                    reinterpret_cast<void *>((uintptr_t)256), (size_t)CAWN_STATIC_SCRATCH_BYTES, st, nullptr, nullptr, 0,
+                    /*validate_only=*/true);
+    if (rc != CAWN_OK) return rc;
     void *scratch = nullptr;
     if (static_scratch_address(&scratch) != cudaSuccess) return CAWN_ERR_CUDA;
-    cudaStream_t st = (cudaStream_t)cuda_stream;
     WsHeader *ws = reinterpret_cast<WsHeader *>(scratch);
     // the array keeps the previous call's contents: only the sticky status has to start at zero
     if (cudaMemsetAsync(&ws->status, 0, sizeof(unsigned), st) != cudaSuccess) return CAWN_ERR_CUDA;

@@ -33,3 +33,33 @@ def built_libraries():
     older than their sources; a no-op when they are up to date."""
     import __graft_entry__ as entry
     entry.build()
+
+
+def pytest_terminal_summary(terminalreporter, exitstatus, config):
+    """Parity margins of the run: for every test function that compared something, the largest
+    floored error it saw (the quantity the tolerances bound) and the largest unfloored median of
+    the element-wise relative error.  Also written to gpurun_out/parity_margins.json."""
+    import json
+    try:
+        from helpers import MARGINS
+    except Exception:
+        return
+    if not MARGINS:
+        return
+    rows = {}
+    for test, err, med in MARGINS:
+        name = test.split("[")[0]
+        n, e, m = rows.get(name, (0, 0.0, 0.0))
+        rows[name] = (n + 1, max(e, err), max(m, med))
+    terminalreporter.section("parity margins (floored max error | unfloored median error | comparisons)")
+    for name in sorted(rows):
+        n, e, m = rows[name]
+        terminalreporter.write_line("%-96s %.3e  %.3e  %d" % (name, e, m, n))
+    out = os.path.join(ROOT, "gpurun_out")
+    try:
+        os.makedirs(out, exist_ok=True)
+        with open(os.path.join(out, "parity_margins.json"), "w") as f:
+            json.dump({k: {"comparisons": v[0], "floored_max": v[1], "unfloored_median_max": v[2]}
+                       for k, v in sorted(rows.items())}, f, indent=1)
+    except OSError:
+        pass
