@@ -42,7 +42,7 @@ import numpy as np
 
 
 # Kernel launches (and memsets) one call of the multi-launch entry points makes.
-LAUNCHES = {"bwd": 2, "bwd_dynamic": 4, "mixing_bwd": 4, "mixing_bwd_dynamic": 6}
+LAUNCHES = {"bwd": 2, "bwd_dynamic": 2, "mixing_bwd": 2, "mixing_bwd_dynamic": 2}
 
 
 def measured_peak():

@@ -130,6 +130,30 @@ void set_stagger(ScanParams &sp, TileShape ts, int bytes_per_element = 16)
     sp.stagger_slots = 3;
 }
 
+// The backward's epilogue launch: the parameter sums that were asked for and, for the fused path,
+// the rows at the tile seams.  Jobs that are not wanted get no blocks.
+cudaError_t launch_epilogue(EpilogueParams ep, bool want_q, bool want_s, bool want_c, bool want_seams, cudaStream_t st)
+{
+    ep.nb_q = want_q ? (ep.C + kEpiCW - 1) / kEpiCW : 0;
+    ep.nb_s = want_s ? (ep.F + kEpiFW - 1) / kEpiFW : 0;
+    ep.nb_c = want_c ? (ep.C + kEpiCW - 1) / kEpiCW : 0;
+    ep.nb_ex = (ep.C + kEpiWarps * 32 - 1) / (kEpiWarps * 32);
+    const long long seams = want_seams ? (long long)ep.nb_ex * (ep.K + 1) * ep.B : 0;
+    const long long blocks = (long long)ep.nb_q + ep.nb_s + ep.nb_c + seams;
+    if (blocks == 0) return cudaSuccess;
+    if (blocks > 2147483647ll) return cudaErrorInvalidValue;
+    cawn_bwd_epilogue_kernel<<<(unsigned)blocks, kEpiWarps * 32, 0, st>>>(ep);
+    return cudaGetLastError();
+}
+
+// The logit gradient of a (row, head) is complete inside one 64-channel group when the group holds
+// whole heads: it is then stored, not accumulated, and needs no zeroing first.
+inline bool logit_grad_direct(const cawn_params *p)
+{
+    const long long C = (long long)p->H * p->F;
+    return C <= 64 || (p->F <= 64 && 64 % p->F == 0);
+}
+
 constexpr uint32_t kBf16Flags = CAWN_FLAG_INPUT_BF16 | CAWN_FLAG_OUTPUT_BF16;
 inline int io_of(const cawn_params *p)
 {
@@ -451,8 +475,9 @@ static int bwd_common(const cawn_params *params, bool dyn, const void *saved, in
         if (grad_fbias && cudaMemsetAsync(grad_fbias, 0, params->F * sizeof(float), st) != cudaSuccess) return CAWN_ERR_CUDA;
         return CAWN_OK;
     }
-    // the logit gradient is accumulated with atomic adds: it starts from zero
-    if (grad_logit != nullptr &&
+    // where the logit gradient is accumulated with atomic adds it starts from zero
+    const bool direct = logit_grad_direct(params);
+    if (grad_logit != nullptr && !direct &&
         cudaMemsetAsync(grad_logit, 0, (size_t)params->B * (size_t)params->L * params->H * sizeof(float), st) != cudaSuccess)
         return CAWN_ERR_CUDA;
 
@@ -499,19 +524,18 @@ static int bwd_common(const cawn_params *params, bool dyn, const void *saved, in
     sp.poll_limit = kPollLimit;
     sp.gamma_logit = gamma_logit; sp.freq_bias = freq_bias; sp.H = params->H; sp.F = params->F;
     sp.grad_logit = (dyn && want_param) ? grad_logit : nullptr;
+    sp.logit_direct = direct ? 1 : 0;
     sp.spart = (dyn && want_param && grad_fbias != nullptr) ? spart : nullptr;
     if (launch_bwd(tb, sp, st, dyn) != cudaSuccess) return CAWN_ERR_CUDA;
 
     if (want_param) {
-        const int warps = 8;
-        cawn_bwd_finalize_kernel<<<(C + warps - 1) / warps, warps * 32, 0, st>>>(
-            qpart, params->B * gb.K, C, dyn ? nullptr : gamma, theta, dyn ? nullptr : grad_gamma, grad_theta, sp.clampv);
-        if (cudaGetLastError() != cudaSuccess) return CAWN_ERR_CUDA;
-        if (dyn && grad_fbias != nullptr) {
-            cawn_bwd_freq_bias_kernel<<<(params->F + warps - 1) / warps, warps * 32, 0, st>>>(
-                spart, params->B * gb.K, params->H, params->F, grad_fbias);
-            if (cudaGetLastError() != cudaSuccess) return CAWN_ERR_CUDA;
-        }
+        EpilogueParams ep;
+        memset(&ep, 0, sizeof(ep));
+        ep.nparts = params->B * gb.K; ep.C = C; ep.H = params->H; ep.F = params->F;
+        ep.qpart = qpart; ep.gamma = dyn ? nullptr : gamma; ep.theta = theta;
+        ep.grad_gamma = dyn ? nullptr : grad_gamma; ep.grad_theta = grad_theta; ep.clampv = sp.clampv;
+        ep.spart = spart; ep.grad_fbias = grad_fbias;
+        if (launch_epilogue(ep, true, dyn && grad_fbias != nullptr, false, false, st) != cudaSuccess) return CAWN_ERR_CUDA;
     }
     return CAWN_OK;
 }
@@ -591,8 +615,9 @@ static int mix_bwd_common(const cawn_params *params, bool dyn, const float *h, c
         if (grad_fbias && cudaMemsetAsync(grad_fbias, 0, (size_t)params->F * sizeof(float), st) != cudaSuccess) return CAWN_ERR_CUDA;
         return CAWN_OK;
     }
-    // the logit gradient is accumulated with atomic adds: it starts from zero
-    if (grad_logit != nullptr &&
+    // where the logit gradient is accumulated with atomic adds it starts from zero
+    const bool direct = logit_grad_direct(params);
+    if (grad_logit != nullptr && !direct &&
         cudaMemsetAsync(grad_logit, 0, (size_t)params->B * (size_t)params->L * params->H * sizeof(float), st) != cudaSuccess)
         return CAWN_ERR_CUDA;
 
@@ -627,6 +652,7 @@ static int mix_bwd_common(const cawn_params *params, bool dyn, const float *h, c
     sp.H = params->H; sp.F = params->F;
     sp.gamma_logit = gamma_logit; sp.freq_bias = freq_bias;
     sp.grad_logit = (dyn && want_scan_param) ? grad_logit : nullptr;
+    sp.logit_direct = direct ? 1 : 0;
     sp.spart = (dyn && want_scan_param && grad_fbias != nullptr) ? spart : nullptr;
     sp.hid = h; sp.conv_w = conv_w; sp.conv_bias = conv_bias; sp.tail_in = tail_in;
     sp.conv_k = Kc;
@@ -636,30 +662,19 @@ static int mix_bwd_common(const cawn_params *params, bool dyn, const float *h, c
     sp.cpart = want_conv_param ? cpart : nullptr;
     if ((dyn ? launch_mix_bwd_dynamic(ts, sp, st) : launch_mix_bwd(ts, sp, st)) != cudaSuccess) return CAWN_ERR_CUDA;
 
-    // 2. rows at the tile seams and the gradient of the carried conv history
-    {
-        const dim3 grid((unsigned)((C + 127) / 128), (unsigned)(g.K + 1), (unsigned)params->B);
-        cawn_mix_bwd_edges_kernel<<<grid, 128, 0, st>>>(edge, conv_w, dtail_out, grad_h, dtail_in, params->L, params->B,
-                                                         C, g.K, ts.T * ts.W, Kc);
-        if (cudaGetLastError() != cudaSuccess) return CAWN_ERR_CUDA;
-    }
-    // 3. parameter gradients from the per-tile partial sums
-    const int warps = 8;
-    if (want_scan_param) {
-        cawn_bwd_finalize_kernel<<<(C + warps - 1) / warps, warps * 32, 0, st>>>(
-            qpart, params->B * g.K, C, dyn ? nullptr : gamma, theta, dyn ? nullptr : grad_gamma, grad_theta, sp.clampv);
-        if (cudaGetLastError() != cudaSuccess) return CAWN_ERR_CUDA;
-        if (dyn && grad_fbias != nullptr) {
-            cawn_bwd_freq_bias_kernel<<<(params->F + warps - 1) / warps, warps * 32, 0, st>>>(
-                spart, params->B * g.K, params->H, params->F, grad_fbias);
-            if (cudaGetLastError() != cudaSuccess) return CAWN_ERR_CUDA;
-        }
-    }
-    if (want_conv_param) {
-        cawn_conv_grad_finalize_kernel<<<(C + warps - 1) / warps, warps * 32, 0, st>>>(
-            cpart, params->B * g.K, C, Kc, grad_conv_w, grad_conv_bias);
-        if (cudaGetLastError() != cudaSuccess) return CAWN_ERR_CUDA;
-    }
+    // 2. one more launch: the rows at the tile seams, the gradient of the carried conv history, and
+    //    the parameter gradients from the per-tile partial sums
+    EpilogueParams ep;
+    memset(&ep, 0, sizeof(ep));
+    ep.nparts = params->B * g.K; ep.C = C; ep.H = params->H; ep.F = params->F; ep.Kc = Kc;
+    ep.qpart = qpart; ep.gamma = dyn ? nullptr : gamma; ep.theta = theta;
+    ep.grad_gamma = dyn ? nullptr : grad_gamma; ep.grad_theta = grad_theta; ep.clampv = sp.clampv;
+    ep.spart = spart; ep.grad_fbias = grad_fbias;
+    ep.cpart = cpart; ep.grad_w = grad_conv_w; ep.grad_bias = grad_conv_bias;
+    ep.edge_du = edge; ep.conv_w = conv_w; ep.dtail_out = dtail_out; ep.grad_h = grad_h; ep.dtail_in = dtail_in;
+    ep.L = params->L; ep.B = params->B; ep.K = g.K; ep.tile = ts.T * ts.W;
+    if (launch_epilogue(ep, want_scan_param, dyn && want_scan_param && grad_fbias != nullptr, want_conv_param, true, st) != cudaSuccess)
+        return CAWN_ERR_CUDA;
     return CAWN_OK;
 }
 

@@ -150,8 +150,10 @@ __device__ __forceinline__ float4 scale_step2(float4 a, float4 P, float2 g, floa
     return make_float4(fmaf(g.x, t.x, x.x), fmaf(g.x, t.y, x.y), fmaf(g.y, t.z, x.z), fmaf(g.y, t.w, x.w));
 }
 // Single-instruction special functions in their flush-to-zero forms (no subnormal fix-up code
-// around them).  Callers keep arguments and results in the normal range: ex2 of |x| <= 40,
-// reciprocals of values in [1, 1e25], sines and cosines of |x| <= pi whose results only feed sums.
+// around them).  What the callers rely on: ex2 of a large argument is +inf and of a very negative
+// one +0, the reciprocal of +inf is +0 and of 1 is 1 (the limits of the sigmoid and tanh forms
+// built from them); sines and cosines are taken of angles in [0, 2 pi] or [-pi, pi], where the
+// approximation's absolute error (about 2^-21) is far below the tolerance, and only feed sums.
 __device__ __forceinline__ float ex2_ftz(float x)
 {
     float y;

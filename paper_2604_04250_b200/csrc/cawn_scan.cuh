@@ -108,7 +108,10 @@ struct ScanParams {
     const float *gamma_logit;    // [B][L][H]
     const float *freq_bias;      // [F]
     int H, F;
-    float *grad_logit;           // BWD: [B][L][H], zeroed before the launch (atomic adds)
+    float *grad_logit;           // BWD: [B][L][H]
+    int logit_direct;            // every 64-channel group holds whole heads: the logit gradient of a (row, head)
+                                 // is complete in one warp and is stored; otherwise it is added atomically
+                                 // into an array zeroed before the launch
     float *spart;                // BWD: per-tile partial sums of the logit gradient [B*K][C]
     // First-wave stagger: the CTAs that land in the 2nd, 3rd, ... resident slot of an SM (linear
     // block index / stagger_group) start their copies stagger_cycles, 2 stagger_cycles, ... late,
@@ -578,23 +581,14 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
         const int Kc = prm.conv_k;
         // the first group of rows (and the history) has landed: the rolling window of the conv
         if (fused_tail_group) cp_async_wait_all(); else cp_async_wait_pending(NG - 1);
-        float2 hv0 = hidden_row(0), hv1 = hidden_row(1), hv2 = hidden_row(2), hv3, hq[GR];
+        float2 hv0 = hidden_row(0), hv1 = hidden_row(1), hv2 = hidden_row(2), hq[GR];
         const bool act = prm.clamp_silu != 0;
         const float tau = prm.gate_tau;
-        const bool want_mask = prm.mask != nullptr;
+        const bool want_mask = MASKED && prm.mask != nullptr;
         uint32_t *const mrow0 = prm.mask + ((long long)b * L + s0) * prm.MW + g * 2;
         unsigned mkeep = 0u;                              // lane r: word 0 of row r; lane 16 + r: word 1
         const bool second_word = g * 2 + 1 < prm.MW;
-        // All of it runs two channels wide on packed fp32 pairs (fma.rn.f32x2 and friends): a
-        // lane's hidden values already come as (channel, channel+1) pairs, and the pushes are
-        // kept in shared memory as (re, re, im, im) so that the scan stays two wide as well.
-        float2 w2[4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) w2[j] = make_float2(wA[j], wB[j]);
-        const float2 b2 = make_float2(bA, bB);
-        const float2 ar2 = make_float2(a.x, a.z), ai2 = make_float2(a.y, a.w), nai2 = make_float2(-a.y, -a.w);
-        const float2 one2 = make_float2(1.f, 1.f);
-        float2 er2 = make_float2(0.f, 0.f), ei2 = er2;
+        const bool tap0 = Kc >= 4, tap1 = Kc >= 3, tap2 = Kc >= 2;
         // DYN: the rows' retention logits, all requested up front so that their latencies overlap
         float2 lgf[DYN ? T : 1];
         if constexpr (DYN) {
@@ -608,80 +602,77 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
                 }
             }
         }
-#pragma unroll
-        for (int i = 0; i < T; ++i) {
-            if (i % GR == 0) {
-                // the group's GR new hidden rows come out of the slice together, then the warp
-                // synchronises once: the pushes of these GR steps only reach rows read by now
-                if (i > 0 && !fused_tail_group) cp_async_wait_pending(NG - 1 - i / GR);
-#pragma unroll
-                for (int q = 0; q < GR; ++q) hq[q] = hidden_row(i + kHalo + q);
-                __syncwarp();
-            }
-            hv3 = hq[i % GR];
-            float2 u = b2;
-            if (0 >= 4 - Kc) u = __ffma2_rn(w2[0], hv0, u);               // fmaf per channel, tap order
-            if (1 >= 4 - Kc) u = __ffma2_rn(w2[1], hv1, u);
-            if (2 >= 4 - Kc) u = __ffma2_rn(w2[2], hv2, u);
-            u = __ffma2_rn(w2[3], hv3, u);
-            hv0 = hv1; hv1 = hv2; hv2 = hv3;
-            float2 x = u;
+        // One channel's push from its conv output u.  With q = e^-x: m = 1/(1+q) and
+        // tanh x = 2/(1+q^2) - 1, so the phase is 2 pi r - pi with r = 1/(1+q^2), and
+        // (cos, sin)(2 pi r - pi) = -(cos, sin)(2 pi r): z = -m (cos, sin)(2 pi r).  A q that
+        // overflows to +inf gives m = 0 and r = 0, a q that underflows gives m = 1 and r = 1: the right
+        // limits, without any clamp on the exponent.
+        auto push = [&](float u, bool valid, float &zr, float &zi) -> bool {
+            float x = u;
             if (act) {
-                x.x = fminf(fmaxf(x.x, -50.f), 50.f); x.y = fminf(fmaxf(x.y, -50.f), 50.f);
-                x.x = __fdividef(x.x, 1.f + __expf(-x.x)); x.y = __fdividef(x.y, 1.f + __expf(-x.y));
+                x = fminf(fmaxf(x, -50.f), 50.f);
+                x = __fdividef(x, 1.f + __expf(-x));
             }
-            // one exponential serves both maps: with q = e^-x, sigmoid = 1/(1+q) and
-            // tanh = (1-q^2)/(1+q^2); |x| is capped where both have long saturated in fp32
-            // q = e^-x as 2^(-x log2 e): the clamp bounds carry the factor
-            const float2 xl = __fmul2_rn(x, make_float2(-1.44269504088896f, -1.44269504088896f));
-            const float2 q = make_float2(ex2_ftz(fminf(fmaxf(xl.x, -36.f), 36.f)), ex2_ftz(fminf(fmaxf(xl.y, -36.f), 36.f)));
-            const float2 q2 = __fmul2_rn(q, q);
-            const float2 p1 = __fadd2_rn(q, one2), p2 = __fadd2_rn(q2, one2);
-            const float2 den = __fmul2_rn(p1, p2);
-            const float2 rcp = make_float2(rcp_ftz(den.x), rcp_ftz(den.y));
-            float2 m = __fmul2_rn(p2, rcp);
-            const float2 n1 = __ffma2_rn(q, make_float2(-q.x, -q.y), one2);
-            const float2 ang = __fmul2_rn(__fmul2_rn(__fmul2_rn(n1, p1), rcp), make_float2(3.14159265358979f, 3.14159265358979f));
-            float2 cs, sn;
-            sincos_ftz(ang.x, sn.x, cs.x);
-            sincos_ftz(ang.y, sn.y, cs.y);
+            const float q = ex2_ftz(x * -1.44269504088896f);
+            const float m = rcp_ftz(1.f + q);
+            const float r = rcp_ftz(fmaf(q, q, 1.f));
+            float sn, cs;
+            sincos_ftz(r * 6.28318530717959f, sn, cs);
             // with clamp + SiLU the magnitude never falls below 0.43, and the host only admits
             // thresholds under that: every gate is open
-            const bool oA = vA && (act || u.x >= tau), oB = vB && (act || u.y >= tau);
-            m.x = oA ? m.x : 0.f; m.y = oB ? m.y : 0.f;
-            const float2 zr = __fmul2_rn(m, cs), zi = __fmul2_rn(m, sn);
-            xs[i * 32] = make_float4(zr.x, zr.y, zi.x, zi.y);            // (re, re, im, im)
-            if (want_mask) {
-                const unsigned bits = ((oA ? 1u : 0u) | (oB ? 2u : 0u)) << (2 * (lane & 15));
-                const unsigned w0 = __reduce_or_sync(0xffffffffu, lane < 16 ? bits : 0u);
-                const unsigned w1 = __reduce_or_sync(0xffffffffu, lane < 16 ? 0u : bits);
-                // rows are parked in lanes and stored sixteen at a time
-                if (lane == (i & 15)) mkeep = w0;
-                if (lane == 16 + (i & 15)) mkeep = w1;
-                if ((i & 15) == 15 || i == T - 1) {
-                    const int r = i - (i & 15) + (lane & 15);
-                    if ((lane & 15) <= (i & 15) && (FULL || r < nvalid) && (lane < 16 || second_word))
-                        mrow0[(long long)r * prm.MW + (lane >> 4)] = mkeep;
+            const bool open = valid && (act || u >= tau);
+            const float mn = open ? -m : 0.f;
+            zr = mn * cs; zi = mn * sn;
+            return open;
+        };
+#pragma unroll
+        for (int gi = 0; gi < NG; ++gi) {
+            // the group's GR new hidden rows come out of the slice together, then the warp
+            // synchronises once: the pushes of these GR steps only reach rows read by now
+            if (gi > 0 && !fused_tail_group) cp_async_wait_pending(NG - 1 - gi);
+#pragma unroll
+            for (int q = 0; q < GR; ++q) hq[q] = hidden_row(gi * GR + kHalo + q);
+            __syncwarp();
+#pragma unroll
+            for (int q = 0; q < GR; ++q) {
+                const int i = gi * GR + q;
+                const float2 hv3 = hq[q];
+                float uA = bA, uB = bB;
+                if (tap0) { uA = fmaf(wA[0], hv0.x, uA); uB = fmaf(wB[0], hv0.y, uB); }     // fmaf per channel, tap order
+                if (tap1) { uA = fmaf(wA[1], hv1.x, uA); uB = fmaf(wB[1], hv1.y, uB); }
+                if (tap2) { uA = fmaf(wA[2], hv2.x, uA); uB = fmaf(wB[2], hv2.y, uB); }
+                uA = fmaf(wA[3], hv3.x, uA); uB = fmaf(wB[3], hv3.y, uB);
+                hv0 = hv1; hv1 = hv2; hv2 = hv3;
+                float4 z;
+                const bool oA = push(uA, vA, z.x, z.y), oB = push(uB, vB, z.z, z.w);
+                xs[i * 32] = z;
+                if (want_mask) {
+                    const unsigned bits = ((oA ? 1u : 0u) | (oB ? 2u : 0u)) << (2 * (lane & 15));
+                    const unsigned w0 = __reduce_or_sync(0xffffffffu, lane < 16 ? bits : 0u);
+                    const unsigned w1 = __reduce_or_sync(0xffffffffu, lane < 16 ? 0u : bits);
+                    // rows are parked in lanes and stored sixteen at a time
+                    if (lane == (i & 15)) mkeep = w0;
+                    if (lane == 16 + (i & 15)) mkeep = w1;
+                    if ((i & 15) == 15 || i == T - 1) {
+                        const int r = i - (i & 15) + (lane & 15);
+                        if ((lane & 15) <= (i & 15) && (FULL || r < nvalid) && (lane < 16 || second_word))
+                            mrow0[(long long)r * prm.MW + (lane >> 4)] = mkeep;
+                    }
                 }
-            }
-            if (FULL || i < nvalid) {
-                if constexpr (DYN) {
-                    // e <- gamma_t (a e) + z, the factor pair kept for phase 3
-                    const float2 gm = make_float2(vA ? sigmoidf_fast(lgf[i].x + fbA) : 0.f,
-                                                  vB ? sigmoidf_fast(lgf[i].y + fbB) : 0.f);
-                    sm.sG[w * T + i][lane] = gm;
-                    dprod.x *= gm.x; dprod.y *= gm.y;
-                    const float2 tr = __ffma2_rn(ar2, er2, __fmul2_rn(nai2, ei2));
-                    const float2 ti = __ffma2_rn(ar2, ei2, __fmul2_rn(ai2, er2));
-                    er2 = __ffma2_rn(gm, tr, zr); ei2 = __ffma2_rn(gm, ti, zi);
-                } else {
-                    const float2 nr = __ffma2_rn(ar2, er2, __ffma2_rn(nai2, ei2, zr));
-                    const float2 ni = __ffma2_rn(ar2, ei2, __ffma2_rn(ai2, er2, zi));
-                    er2 = nr; ei2 = ni;
+                if (FULL || i < nvalid) {
+                    if constexpr (DYN) {
+                        // e <- gamma_t (a e) + z, the factor pair kept for phase 3
+                        const float2 gm = make_float2(vA ? sigmoidf_fast(lgf[i].x + fbA) : 0.f,
+                                                      vB ? sigmoidf_fast(lgf[i].y + fbB) : 0.f);
+                        sm.sG[w * T + i][lane] = gm;
+                        dprod.x *= gm.x; dprod.y *= gm.y;
+                        e = scale_step2(a, e, gm, z);
+                    } else {
+                        e = cfma2(a, e, z);
+                    }
                 }
             }
         }
-        e = make_float4(er2.x, ei2.x, er2.y, ei2.y);
     } else if constexpr (KIND == KIND_FWD) {
         // |p| >= eps decided as re^2 + im^2 >= eps^2 in double: both squares are exact there
         // and the sum rounds once, so the decision is reproducible bit for bit.  The fp32 sum
@@ -1055,8 +1046,10 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
                                     float v = (vA && hA == h ? sA : 0.f) + (vB && hB == h ? sB : 0.f);
 #pragma unroll
                                     for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
-                                    if (lane == 0)
-                                        atomicAdd(prm.grad_logit + ((long long)b * L + (t_first - i)) * prm.H + h, v);
+                                    if (lane == 0) {
+                                        float *gl = prm.grad_logit + ((long long)b * L + (t_first - i)) * prm.H + h;
+                                        if (prm.logit_direct) *gl = v; else atomicAdd(gl, v);
+                                    }
                                 }
                             }
                         }
@@ -1069,32 +1062,7 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
                 }
             }
         };
-        if constexpr (KIND == KIND_FUSED) {
-            // the pushes sit in shared memory as (re, re, im, im): the recurrence runs two wide
-            const float2 ar2 = make_float2(a.x, a.z), ai2 = make_float2(a.y, a.w), nai2 = make_float2(-a.y, -a.w);
-            float2 Pr = make_float2(P.x, P.z), Pi = make_float2(P.y, P.w);
-#pragma unroll
-            for (int i = 0; i < T; ++i) {
-                if (FULL || i < nvalid) {
-                    const float4 z = xs[i * 32];
-                    if constexpr (DYN) {
-                        gstep = sm.sG[w * T + i][lane];
-                        const float2 tr = __ffma2_rn(ar2, Pr, __fmul2_rn(nai2, Pi));
-                        const float2 ti = __ffma2_rn(ar2, Pi, __fmul2_rn(ai2, Pr));
-                        Pr = __ffma2_rn(gstep, tr, make_float2(z.x, z.y));
-                        Pi = __ffma2_rn(gstep, ti, make_float2(z.z, z.w));
-                    } else {
-                        const float2 nr = __ffma2_rn(ar2, Pr, __ffma2_rn(nai2, Pi, make_float2(z.x, z.y)));
-                        const float2 ni = __ffma2_rn(ar2, Pi, __ffma2_rn(ai2, Pr, make_float2(z.z, z.w)));
-                        Pr = nr; Pi = ni;
-                    }
-                    float4 o = make_float4(Pr.x, Pi.x, Pr.y, Pi.y);
-                    if (cl > 0.f) o = clamp4(o, cl);
-                    store_row(i, o);
-                }
-            }
-            P = make_float4(Pr.x, Pi.x, Pr.y, Pi.y);
-        } else if (cl > 0.f) {
+        if (cl > 0.f) {
 #pragma unroll
             for (int i = 0; i < T; ++i) step_row(i, true);
         } else {
@@ -1121,8 +1089,10 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
                 for (int off = 16 / T; off >= 1; off >>= 1) rowsum[0] += __shfl_xor_sync(0xffffffffu, rowsum[0], off);
                 constexpr int LPR = 32 / T;              // lanes per row
                 const int row = lane / LPR;
-                if (lane % LPR == 0 && (FULL || row < nvalid))
-                    atomicAdd(prm.grad_logit + ((long long)b * L + (t_first - row)) * prm.H + h_lo, rowsum[0]);
+                if (lane % LPR == 0 && (FULL || row < nvalid)) {
+                    float *gl = prm.grad_logit + ((long long)b * L + (t_first - row)) * prm.H + h_lo;
+                    if (prm.logit_direct) *gl = rowsum[0]; else atomicAdd(gl, rowsum[0]);
+                }
             }
         }
         // An Inf or NaN that entered anywhere (an input, the carried state, an overflow) is still

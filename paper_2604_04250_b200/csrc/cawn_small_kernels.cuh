@@ -5,54 +5,192 @@
 
 namespace cawn {
 
-// grad_gamma_j = Re(e^{i theta} Q_j), grad_theta_j = -Im(a_j Q_j), Q_j = sum of the per-tile
-// partials in a fixed order, in double.  One warp per channel.
-__global__ void cawn_bwd_finalize_kernel(const float2 *qpart, int nparts, int C,
-                                         const float *gamma, const float *theta,
-                                         float *grad_gamma, float *grad_theta, float clampv)
+// ---------------------------------------------------------------------------------------
+// The backward's epilogue launch: everything that has to wait for the whole reverse scan, in one
+// kernel.  A block does one of four jobs, chosen by its index:
+//   [0, nb_q)            grad_gamma_j = Re(e^{i theta} Q_j), grad_theta_j = -Im(a_j Q_j), Q_j = sum of the
+//                        per-tile partials qpart [nparts][C]; 8 channels per block
+//   [nb_q, +nb_s)        time-varying retention: grad_freq_bias[k] = sum over tiles and heads of spart
+//                        [nparts][C]; 2 harmonics per block
+//   [.., +nb_c)          fused path: grad_conv_w[c][k], grad_conv_bias[c] from cpart [nparts][C][5];
+//                        8 channels per block
+//   the rest             fused path: grad_h of the rows at tile seams and the gradient of the carried conv
+//                        history, from edge_du (see seam_rows below); one thread per channel
+// Sums run in double in a fixed order.  A block owns CW adjacent channels; a lane is (sub, channel) =
+// (lane / CW, lane % CW), so a warp load covers 32 / CW parts with CW contiguous channels each, and
+// thread (warp w, sub) takes parts (w * 32 / CW + sub) + i * kEpiWarps * 32 / CW.  The warps' sums are added in
+// warp order, then the subs' by a butterfly (both partners of an exchange form the same sum).
+// Bitwise repeatable.
+constexpr int kEpiWarps = 32;
+constexpr int kEpiCW = 8;            // channels per block of the q and c jobs
+constexpr int kEpiFW = 2;            // harmonics per block of the s job
+struct EpilogueParams {
+    int nb_q, nb_s, nb_c, nb_ex;     // blocks per job; nb_ex: blocks along the channels of one seam
+    int nparts, C, H, F, Kc;
+    const float2 *qpart;
+    const float *gamma, *theta;      // gamma NULL: time-varying retention (the factor is already in Q)
+    float *grad_gamma, *grad_theta;
+    float clampv;
+    const float *spart;
+    float *grad_fbias;
+    const float *cpart;
+    float *grad_w, *grad_bias;
+    const float *edge_du, *conv_w, *dtail_out;
+    float *grad_h, *dtail_in;
+    long long L;
+    int B, K, tile;
+};
+
+// Sum of NV doubles per thread over the block: first over the warps, lane by lane, in warp order,
+// then over the lanes that hold the same channel (lanes CW apart).  Result valid in warp 0.
+template <int NV, int CW>
+__device__ __forceinline__ void block_sum_fixed_order(double (&v)[NV], double *sh)
 {
-    const int lane = threadIdx.x & 31;
-    const int ch = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    if (ch >= C) return;
-    double sr = 0.0, si = 0.0;
-    for (int p = lane; p < nparts; p += 32) {
-        const float2 q = qpart[(long long)p * C + ch];
-        sr += (double)q.x;
-        si += (double)q.y;
-    }
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
 #pragma unroll
-    for (int off = 16; off > 0; off >>= 1) {
-        sr += __shfl_down_sync(0xffffffffu, sr, off);
-        si += __shfl_down_sync(0xffffffffu, si, off);
-    }
-    if (lane == 0) {
-        const double gm = gamma != nullptr ? (double)gamma[ch] : 1.0;   // time-varying: already in Q
-        double sn, cs;
-        sincos((double)theta[ch], &sn, &cs);
-        double dg = cs * sr - sn * si;
-        const double dth = -gm * (cs * si + sn * sr);
-        if (clampv > 0.f) dg = fmin(fmax(dg, -(double)clampv), (double)clampv);
-        if (grad_gamma != nullptr) grad_gamma[ch] = (float)dg;
-        if (grad_theta != nullptr) grad_theta[ch] = (float)dth;
+    for (int j = 0; j < NV; ++j) sh[(w * NV + j) * 32 + lane] = v[j];
+    __syncthreads();
+    if (w == 0) {
+#pragma unroll
+        for (int j = 0; j < NV; ++j) {
+            double acc = sh[j * 32 + lane];
+            for (int i = 1; i < kEpiWarps; ++i) acc += sh[(i * NV + j) * 32 + lane];
+#pragma unroll
+            for (int off = CW; off < 32; off <<= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+            v[j] = acc;
+        }
     }
 }
 
-// Time-varying retention: grad_freq_bias[k] = sum over tiles and heads of the per-channel
-// partial sums of the logit gradient, in a fixed order, in double.  One warp per harmonic.
-__global__ void cawn_bwd_freq_bias_kernel(const float *spart, int nparts, int H, int F, float *grad_freq_bias)
+// Backward of the fused path, rows at tile seams.  The scan kernel (KIND_MIXBWD) leaves out
+// grad_h of the three last rows in time of every tile, whose conv transpose reaches into the
+// tile after them, and stores every tile's du at both ends instead (edge_du [B*K][6][C]: rows
+// t_hi, t_hi-1, t_hi-2, then t_lo, t_lo+1, t_lo+2; tiles are counted from the END of the call:
+// tile k covers t_hi = L-1-k*tile down to t_lo = max(L-(k+1)*tile, 0)).  Here:
+//   grad_h(s) = sum_j w[j] du(s + 3 - j) (+ the incoming gradient of the conv history on the
+//   call's last conv_k-1 rows)          for those rows (kb < K), and
+//   grad of the carried history rows s = -Kh .. -1 (kb = K), which collect from du(0..2)
+//   and, when the call is shorter than the history, pass part of the incoming gradient through.
+// One thread per channel; taps right-aligned as in the scan kernel.
+__device__ __forceinline__ void seam_rows(const EpilogueParams &ep, int c, int kb, int b)
 {
-    const int lane = threadIdx.x & 31;
-    const int kf = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    if (kf >= F) return;
-    const long long C = (long long)H * F;
-    double acc = 0.0;
-    for (long long i = lane; i < (long long)nparts * H; i += 32) {
-        const long long part = i / H, h = i % H;
-        acc += (double)spart[part * C + h * F + kf];
-    }
+    const int C = ep.C, K = ep.K, tile = ep.tile, Kc = ep.Kc, Kh = Kc - 1;
+    const long long L = ep.L;
+    float wt[4];
 #pragma unroll
-    for (int off = 16; off > 0; off >>= 1) acc += __shfl_down_sync(0xffffffffu, acc, off);
-    if (lane == 0) grad_freq_bias[kf] = (float)acc;
+    for (int j = 0; j < 4; ++j) wt[j] = j >= 4 - Kc ? ep.conv_w[(long long)c * Kc + (j - (4 - Kc))] : 0.f;
+    // du at physical row r, from whichever tile end holds it
+    auto DU = [&](long long r) -> float {
+        if (r < 0 || r >= L) return 0.f;
+        const long long kk = (L - 1 - r) / tile;
+        const long long t_hi = L - 1 - kk * tile;
+        long long t_lo = L - (kk + 1) * tile;
+        if (t_lo < 0) t_lo = 0;
+        const float *e = ep.edge_du + (((long long)b * K + kk) * 6) * C + c;
+        if (t_hi - r < 3) return e[(t_hi - r) * C];
+        if (r - t_lo < 3) return e[(3 + (r - t_lo)) * C];
+        return 0.f;                                  // not an edge row: never asked for
+    };
+    if (kb < K) {
+        const long long t_hi = L - 1 - (long long)kb * tile;
+        long long t_lo = L - (long long)(kb + 1) * tile;
+        if (t_lo < 0) t_lo = 0;
+        for (long long s = t_hi; s >= t_lo && s > t_hi - 3; --s) {
+            float acc = 0.f;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) acc = fmaf(wt[j], DU(s + 3 - j), acc);
+            if (ep.dtail_out != nullptr && s >= L - Kh) acc += ep.dtail_out[((long long)b * Kh + (s - (L - Kh))) * C + c];
+            ep.grad_h[((long long)b * L + s) * C + c] = acc;
+        }
+    } else if (ep.dtail_in != nullptr) {
+        for (int r = 0; r < Kh; ++r) {
+            const long long s = r - Kh;
+            float acc = 0.f;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) acc = fmaf(wt[j], DU(s + 3 - j), acc);
+            if (ep.dtail_out != nullptr && r >= L) acc += ep.dtail_out[((long long)b * Kh + (r - L)) * C + c];
+            ep.dtail_in[((long long)b * Kh + r) * C + c] = acc;
+        }
+    }
+}
+
+__global__ void __launch_bounds__(kEpiWarps * 32) cawn_bwd_epilogue_kernel(const EpilogueParams ep)
+{
+    __shared__ double sh[kEpiWarps * 5 * 32];
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    int blk = blockIdx.x;
+    const int C = ep.C, nparts = ep.nparts;
+    constexpr int PW = 32 / kEpiCW;                   // parts per warp load (q and c jobs)
+    if (blk < ep.nb_q) {
+        const int ch = blk * kEpiCW + lane % kEpiCW;
+        double v[2] = {0.0, 0.0};
+        if (ch < C) {
+#pragma unroll 8
+            for (int p = w * PW + lane / kEpiCW; p < nparts; p += kEpiWarps * PW) {
+                const float2 q = ep.qpart[(long long)p * C + ch];
+                v[0] += (double)q.x;
+                v[1] += (double)q.y;
+            }
+        }
+        block_sum_fixed_order<2, kEpiCW>(v, sh);
+        if (w == 0 && lane < kEpiCW && ch < C) {
+            const double gm = ep.gamma != nullptr ? (double)ep.gamma[ch] : 1.0;   // time-varying: already in Q
+            double sn, cs;
+            sincos((double)ep.theta[ch], &sn, &cs);
+            double dg = cs * v[0] - sn * v[1];
+            const double dth = -gm * (cs * v[1] + sn * v[0]);
+            if (ep.clampv > 0.f) dg = fmin(fmax(dg, -(double)ep.clampv), (double)ep.clampv);
+            if (ep.grad_gamma != nullptr) ep.grad_gamma[ch] = (float)dg;
+            if (ep.grad_theta != nullptr) ep.grad_theta[ch] = (float)dth;
+        }
+        return;
+    }
+    blk -= ep.nb_q;
+    if (blk < ep.nb_s) {
+        // the (part, head) pairs are the terms: pair q = p * H + h holds harmonic kf at spart[p * C + h * F + kf]
+        constexpr int QW = 32 / kEpiFW;
+        const int kf = blk * kEpiFW + lane % kEpiFW;
+        const long long npairs = (long long)nparts * ep.H;
+        double v[1] = {0.0};
+        if (kf < ep.F) {
+#pragma unroll 8
+            for (long long q = w * QW + lane / kEpiFW; q < npairs; q += kEpiWarps * QW) {
+                const long long p = q / ep.H, h = q - p * ep.H;
+                v[0] += (double)ep.spart[p * C + h * ep.F + kf];
+            }
+        }
+        block_sum_fixed_order<1, kEpiFW>(v, sh);
+        if (w == 0 && lane < kEpiFW && kf < ep.F) ep.grad_fbias[kf] = (float)v[0];
+        return;
+    }
+    blk -= ep.nb_s;
+    if (blk < ep.nb_c) {
+        // per-tile partials [nparts][C][5]: four right-aligned taps, then the bias
+        const int ch = blk * kEpiCW + lane % kEpiCW;
+        double v[5] = {0.0, 0.0, 0.0, 0.0, 0.0};
+        if (ch < C) {
+#pragma unroll 4
+            for (int p = w * PW + lane / kEpiCW; p < nparts; p += kEpiWarps * PW) {
+                const float *q = ep.cpart + ((long long)p * C + ch) * 5;
+#pragma unroll
+                for (int j = 0; j < 5; ++j) v[j] += (double)q[j];
+            }
+        }
+        block_sum_fixed_order<5, kEpiCW>(v, sh);
+        if (w == 0 && lane < kEpiCW && ch < C) {
+            if (ep.grad_w != nullptr)
+                for (int k = 0; k < ep.Kc; ++k) ep.grad_w[(long long)ch * ep.Kc + k] = (float)v[k + (4 - ep.Kc)];
+            if (ep.grad_bias != nullptr) ep.grad_bias[ch] = (float)v[4];
+        }
+        return;
+    }
+    blk -= ep.nb_c;
+    {
+        const int cb = blk % ep.nb_ex, rest = blk / ep.nb_ex;
+        const int kb = rest % (ep.K + 1), b = rest / (ep.K + 1);
+        const int c = cb * (kEpiWarps * 32) + threadIdx.x;
+        if (c < C && b < ep.B) seam_rows(ep, c, kb, b);
+    }
 }
 
 // state_out = a^n * state_prev + state_local with a^n = gamma^n (cos n theta, sin n theta)
@@ -74,87 +212,6 @@ __global__ void cawn_state_carry_kernel(const float2 *prev, const float2 *local,
     o.x = (float)((double)l.x + mag * (pr * cs - pi * sn));
     o.y = (float)((double)l.y + mag * (pr * sn + pi * cs));
     out[idx] = o;
-}
-
-// Backward of the fused path, rows at tile seams.  The scan kernel (KIND_MIXBWD) leaves out
-// grad_h of the three last rows in time of every tile, whose conv transpose reaches into the
-// tile after them, and stores every tile's du at both ends instead (edge_du [B*K][6][C]: rows
-// t_hi, t_hi-1, t_hi-2, then t_lo, t_lo+1, t_lo+2; tiles are counted from the END of the call:
-// tile k covers t_hi = L-1-k*tile down to t_lo = max(L-(k+1)*tile, 0)).  Here:
-//   grad_h(s) = sum_j w[j] du(s + 3 - j) (+ the incoming gradient of the conv history on the
-//   call's last conv_k-1 rows)          for those rows (blockIdx.y = k < K), and
-//   grad of the carried history rows s = -Kh .. -1 (blockIdx.y = K), which collect from du(0..2)
-//   and, when the call is shorter than the history, pass part of the incoming gradient through.
-// One thread per channel; taps right-aligned as in the scan kernel.
-__global__ void cawn_mix_bwd_edges_kernel(const float *edge_du, const float *conv_w, const float *dtail_out,
-                                          float *grad_h, float *dtail_in, long long L, int B, int C, int K,
-                                          int tile, int Kc)
-{
-    const int c = blockIdx.x * blockDim.x + threadIdx.x;
-    const int kb = blockIdx.y, b = blockIdx.z;
-    if (c >= C) return;
-    const int Kh = Kc - 1;
-    float wt[4];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) wt[j] = j >= 4 - Kc ? conv_w[(long long)c * Kc + (j - (4 - Kc))] : 0.f;
-    // du at physical row r, from whichever tile end holds it
-    auto DU = [&](long long r) -> float {
-        if (r < 0 || r >= L) return 0.f;
-        const long long kk = (L - 1 - r) / tile;
-        const long long t_hi = L - 1 - kk * tile;
-        long long t_lo = L - (kk + 1) * tile;
-        if (t_lo < 0) t_lo = 0;
-        const float *e = edge_du + (((long long)b * K + kk) * 6) * C + c;
-        if (t_hi - r < 3) return e[(t_hi - r) * C];
-        if (r - t_lo < 3) return e[(3 + (r - t_lo)) * C];
-        return 0.f;                                  // not an edge row: never asked for
-    };
-    if (kb < K) {
-        const long long t_hi = L - 1 - (long long)kb * tile;
-        long long t_lo = L - (long long)(kb + 1) * tile;
-        if (t_lo < 0) t_lo = 0;
-        for (long long s = t_hi; s >= t_lo && s > t_hi - 3; --s) {
-            float acc = 0.f;
-#pragma unroll
-            for (int j = 0; j < 4; ++j) acc = fmaf(wt[j], DU(s + 3 - j), acc);
-            if (dtail_out != nullptr && s >= L - Kh) acc += dtail_out[((long long)b * Kh + (s - (L - Kh))) * C + c];
-            grad_h[((long long)b * L + s) * C + c] = acc;
-        }
-    } else if (dtail_in != nullptr) {
-        for (int r = 0; r < Kh; ++r) {
-            const long long s = r - Kh;
-            float acc = 0.f;
-#pragma unroll
-            for (int j = 0; j < 4; ++j) acc = fmaf(wt[j], DU(s + 3 - j), acc);
-            if (dtail_out != nullptr && r >= L) acc += dtail_out[((long long)b * Kh + (r - L)) * C + c];
-            dtail_in[((long long)b * Kh + r) * C + c] = acc;
-        }
-    }
-}
-
-// grad_conv_w[c][k] and grad_conv_bias[c] from the per-tile partials [nparts][C][5] (four
-// right-aligned taps, then the bias), in double, fixed order.  One warp per channel.
-__global__ void cawn_conv_grad_finalize_kernel(const float *part, int nparts, int C, int Kc,
-                                               float *grad_w, float *grad_bias)
-{
-    const int lane = threadIdx.x & 31;
-    const int ch = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    if (ch >= C) return;
-    double acc[5] = {0.0, 0.0, 0.0, 0.0, 0.0};
-    for (int p = lane; p < nparts; p += 32) {
-        const float *q = part + ((long long)p * C + ch) * 5;
-#pragma unroll
-        for (int j = 0; j < 5; ++j) acc[j] += (double)q[j];
-    }
-#pragma unroll
-    for (int j = 0; j < 5; ++j)
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1) acc[j] += __shfl_down_sync(0xffffffffu, acc[j], off);
-    if (lane == 0) {
-        if (grad_w != nullptr)
-            for (int k = 0; k < Kc; ++k) grad_w[(long long)ch * Kc + k] = (float)acc[k + (4 - Kc)];
-        if (grad_bias != nullptr) grad_bias[ch] = (float)acc[4];
-    }
 }
 
 // One 32-bit word, stream-ordered (the wait hook of a workspace header).

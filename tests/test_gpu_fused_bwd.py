@@ -78,7 +78,7 @@ def compare(got, ref, L, Kc):
         assert floored_rel_err(got["dh"], ref["dh"], axes=(0, 1)) < TOL
     assert floored_rel_err(got["dstate_in"], ref["dstate_in"]) < TOL
     if Kc > 1:
-        assert floored_rel_err(got["dtail_in"], ref["dtail_in"]) < TOL
+        assert floored_rel_err(got["dtail_in"], ref["dtail_in"], axes=None) < TOL
     for k in ("dw", "dbias", "dgamma", "dtheta"):
         if k in got:
             assert not np.isnan(got[k]).any(), k
@@ -140,7 +140,7 @@ def test_mixing_bwd_config4_full_size():
         ref = reference(sub, cfg.gate_eps)
         assert floored_rel_err(got["dh"][b:b + 1], ref["dh"], axes=(0, 1)) < TOL, b
         assert floored_rel_err(got["dstate_in"][b:b + 1], ref["dstate_in"]) < TOL, b
-        assert floored_rel_err(got["dtail_in"][b:b + 1], ref["dtail_in"]) < TOL, b
+        assert floored_rel_err(got["dtail_in"][b:b + 1], ref["dtail_in"], axes=None) < TOL, b
         for k in sums:
             sums[k] = sums[k] + ref[k].astype(np.float64)
     for k in sums:
@@ -192,4 +192,4 @@ def test_mixing_bwd_with_dynamic_retention(B, L, H, F, Kc):
     assert floored_rel_err(gt.cpu().numpy(), ref["dtheta"]) < TOL
     assert floored_rel_err(dP, ref["dstate_in"]) < TOL
     if Kc > 1:
-        assert floored_rel_err(dtail, ref["dtail_in"]) < TOL
+        assert floored_rel_err(dtail, ref["dtail_in"], axes=None) < TOL
