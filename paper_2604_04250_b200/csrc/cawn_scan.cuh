@@ -244,7 +244,9 @@ __device__ __forceinline__ void fetch_rows(float4 *dst, uint32_t dst_s, const ch
 // with m = sigmoid(x), ph = pi tanh(x), x = u (or SiLU(clamp(u)) with `act`), m_used = m where the
 // gate is open, else 0.  Straight-through gate: the magnitude path ignores the gate
 // (dm = lr cos ph + li sin ph), the phase path is scaled by the gated magnitude.
-// m, tanh, sin and cos are recomputed exactly as the forward computes them.
+// As in the forward: q = e^-x, m = 1/(1+q), r = 1/(1+q^2), tanh x = 2r - 1, and
+// (cos, sin)(ph) = -(cos, sin)(2 pi r); 1 - tanh^2 = 4 r (1 - r).  Where (1+q)(1+q^2) overflows
+// m = r = 0, where q underflows m = r = 1, and every term stays finite.
 __device__ __forceinline__ float prelude_du(float u, float lr, float li, bool act, float tau)
 {
     float x = u, dxdu = 1.f;
@@ -254,16 +256,17 @@ __device__ __forceinline__ float prelude_du(float u, float lr, float li, bool ac
         x = v * sg;
         dxdu = (u >= -50.f && u <= 50.f) ? sg * fmaf(v, 1.f - sg, 1.f) : 0.f;
     }
-    const float q = ex2_ftz(fminf(fmaxf(x * -1.44269504088896f, -36.f), 36.f)), q2 = q * q;
-    const float rcp = rcp_ftz((1.f + q) * (1.f + q2));
-    const float m = (1.f + q2) * rcp;
-    const float th = (1.f - q2) * (1.f + q) * rcp;
-    float sn, cs;
-    sincos_ftz(3.14159265358979f * th, sn, cs);
+    const float q = ex2_ftz(fminf(x * -1.44269504088896f, 60.f));
+    const float p1 = 1.f + q, p2 = fmaf(q, q, 1.f);
+    const float rr = rcp_ftz(p1 * p2);
+    const float m = p2 * rr, r = p1 * rr;
+    float sn, cs;                                    // of 2 pi r: the negated sine and cosine of the phase
+    sincos_ftz(r * 6.28318530717959f, sn, cs);
     const bool open = act || u >= tau;           // with clamp + SiLU every gate is open (see the forward)
-    const float dm = fmaf(lr, cs, li * sn);
-    const float dph = (open ? m : 0.f) * fmaf(li, cs, -lr * sn);
-    const float dx = fmaf(dm * m, 1.f - m, dph * 3.14159265358979f * fmaf(-th, th, 1.f));
+    const float dm = -fmaf(lr, cs, li * sn);
+    const float dph = (open ? m : 0.f) * fmaf(lr, sn, -li * cs);
+    // d ph / dx = pi (1 - tanh^2) = 4 pi r (1 - r);  d m / dx = m (1 - m)
+    const float dx = fmaf(dm * m, 1.f - m, dph * (12.5663706143592f * r) * (1.f - r));
     return dx * dxdu;
 }
 
@@ -604,18 +607,20 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
         }
         // One channel's push from its conv output u.  With q = e^-x: m = 1/(1+q) and
         // tanh x = 2/(1+q^2) - 1, so the phase is 2 pi r - pi with r = 1/(1+q^2), and
-        // (cos, sin)(2 pi r - pi) = -(cos, sin)(2 pi r): z = -m (cos, sin)(2 pi r).  A q that
-        // overflows to +inf gives m = 0 and r = 0, a q that underflows gives m = 1 and r = 1: the right
-        // limits, without any clamp on the exponent.
+        // (cos, sin)(2 pi r - pi) = -(cos, sin)(2 pi r): z = -m (cos, sin)(2 pi r).  Both quotients
+        // come from one reciprocal of (1+q)(1+q^2).  q is capped at 2^60 so that 1+q^2 stays finite;
+        // where the product overflows its reciprocal is +0 and m = r = 0, a q that underflows gives
+        // m = r = 1: the right limits.
         auto push = [&](float u, bool valid, float &zr, float &zi) -> bool {
             float x = u;
             if (act) {
                 x = fminf(fmaxf(x, -50.f), 50.f);
                 x = __fdividef(x, 1.f + __expf(-x));
             }
-            const float q = ex2_ftz(x * -1.44269504088896f);
-            const float m = rcp_ftz(1.f + q);
-            const float r = rcp_ftz(fmaf(q, q, 1.f));
+            const float q = ex2_ftz(fminf(x * -1.44269504088896f, 60.f));
+            const float p1 = 1.f + q, p2 = fmaf(q, q, 1.f);
+            const float rr = rcp_ftz(p1 * p2);               // one reciprocal serves both
+            const float m = p2 * rr, r = p1 * rr;
             float sn, cs;
             sincos_ftz(r * 6.28318530717959f, sn, cs);
             // with clamp + SiLU the magnitude never falls below 0.43, and the host only admits
@@ -986,7 +991,11 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
         // rolling window of hidden rows, and the sums for the conv gradients
         float2 hwin[4] = {};                             // h(t), h(t-1), h(t-2), h(t-3) of the current row
         float caA[5] = {}, caB[5] = {};
+        float2 dwin[3] = {};                             // du of the three rows processed before the current one
+        float2 dfirst[3] = {};                           // du of this thread's first three rows (finished after the barrier)
         const bool mact = prm.clamp_silu != 0;
+        const bool mtap0 = prm.conv_k >= 4, mtap1 = prm.conv_k >= 3, mtap2 = prm.conv_k >= 2;
+        float *const gh = reinterpret_cast<float *>(prm.out);
         if constexpr (MIX) {
 #pragma unroll
             for (int r = 0; r < 3; ++r) hwin[r + 1] = *reinterpret_cast<const float2 *>(&sm.hrev[w * T + r][2 * lane]);
@@ -996,22 +1005,36 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
         auto mix_row = [&](int i, float4 lam) {
             hwin[0] = hwin[1]; hwin[1] = hwin[2]; hwin[2] = hwin[3];
             hwin[3] = *reinterpret_cast<const float2 *>(&sm.hrev[w * T + i + 3][2 * lane]);
-            float uA = mbA, uB = mbB;
-#pragma unroll
-            for (int j = 0; j < 4; ++j)
-                if (j >= 4 - prm.conv_k) { uA = fmaf(mwA[j], hwin[3 - j].x, uA); uB = fmaf(mwB[j], hwin[3 - j].y, uB); }
+            float uA = mbA, uB = mbB;                    // the forward's fmaf chain, tap order
+            if (mtap0) { uA = fmaf(mwA[0], hwin[3].x, uA); uB = fmaf(mwB[0], hwin[3].y, uB); }
+            if (mtap1) { uA = fmaf(mwA[1], hwin[2].x, uA); uB = fmaf(mwB[1], hwin[2].y, uB); }
+            if (mtap2) { uA = fmaf(mwA[2], hwin[1].x, uA); uB = fmaf(mwB[2], hwin[1].y, uB); }
+            uA = fmaf(mwA[3], hwin[0].x, uA); uB = fmaf(mwB[3], hwin[0].y, uB);
             const float duA = vA ? prelude_du(uA, lam.x, lam.y, mact, prm.gate_tau) : 0.f;
             const float duB = vB ? prelude_du(uB, lam.z, lam.w, mact, prm.gate_tau) : 0.f;
-            xs[i * 32] = make_float4(duA, duB, 0.f, 0.f);
+            *reinterpret_cast<float2 *>(&xs[i * 32]) = make_float2(duA, duB);
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 caA[j] = fmaf(duA, hwin[3 - j].x, caA[j]);
                 caB[j] = fmaf(duB, hwin[3 - j].y, caB[j]);
             }
             caA[4] += duA; caB[4] += duB;
+            // Transposed conv: grad_h(t) = sum_j w[j] du(t + 3 - j).  In processing order (row R is
+            // time t_hi - R) that is du of rows R-3 .. R: from the fourth row of a thread on they are
+            // all its own and still in registers; its first three rows wait for the barrier.
+            if (i < 3) {
+                dfirst[i] = make_float2(duA, duB);
+            } else {
+                const float gA = fmaf(mwA[3], duA, fmaf(mwA[2], dwin[0].x, fmaf(mwA[1], dwin[1].x, mwA[0] * dwin[2].x)));
+                const float gB = fmaf(mwB[3], duB, fmaf(mwB[2], dwin[0].y, fmaf(mwB[1], dwin[1].y, mwB[0] * dwin[2].y)));
+                float *o = gh + (e0 - (long long)i * C);
+                if (VEC) { if (vA) __stcs(reinterpret_cast<float2 *>(o), make_float2(gA, gB)); }
+                else { if (vA) __stcs(o, gA); if (vB) __stcs(o + 1, gB); }
+            }
+            dwin[2] = dwin[1]; dwin[1] = dwin[0]; dwin[0] = make_float2(duA, duB);
         };
         auto step_row = [&](int i, bool clamped) {
-            if (MIX && !(FULL || i < nvalid)) xs[i * 32] = zero4();      // no such row: its du is 0
+            if (MIX && !(FULL || i < nvalid)) *reinterpret_cast<float2 *>(&xs[i * 32]) = make_float2(0.f, 0.f);      // no such row: its du is 0
             if (FULL || i < nvalid) {
                 float2 gown = make_float2(0.f, 0.f);
                 if constexpr (DYN) {
@@ -1110,21 +1133,22 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
             if (vB) s[1] = make_float2(P.z, P.w);
         }
         if constexpr (MIX) {
-            // Transposed conv: grad_h(t) = sum_j w[j] du(t + 3 - j).  Row R of the tile (physical
-            // t_hi - R) needs du of rows R-3 .. R; the tile's first three rows would need the tile
-            // after it in time, so their du (and the du of its three earliest rows, for the tile
-            // before it) go to the edge area and a small kernel finishes those rows.
+            // The first three rows of every thread need du of the warp before it; the tile's first
+            // three rows would need the tile after it in time, so their du (and the du of its three
+            // earliest rows, for the tile before it) go to the edge area and the epilogue launch
+            // finishes those rows.
             __syncthreads();
             const float4 (*du)[32] = sm.tile[0];
-            float *const gh = reinterpret_cast<float *>(prm.out);
 #pragma unroll
-            for (int i = 0; i < T; ++i) {
+            for (int i = 0; i < 3 && i < T; ++i) {
                 const int R = w * T + i;
                 if ((FULL || i < nvalid) && R >= 3) {
                     float dA = 0.f, dB = 0.f;
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
-                        const float2 d = *reinterpret_cast<const float2 *>(&du[R - 3 + j][lane]);
+                        // rows of this thread are still in registers, earlier ones come from the tile
+                        const float2 d = (i - 3 + j >= 0) ? dfirst[i - 3 + j >= 0 ? i - 3 + j : 0]
+                                                          : *reinterpret_cast<const float2 *>(&du[R - 3 + j][lane]);
                         dA = fmaf(mwA[j], d.x, dA); dB = fmaf(mwB[j], d.y, dB);
                     }
                     float *o = gh + (e0 - (long long)i * C);
