@@ -247,10 +247,11 @@ __device__ __forceinline__ void fetch_rows(float4 *dst, uint32_t dst_s, const ch
 // As in the forward: q = e^-x, m = 1/(1+q), r = 1/(1+q^2), tanh x = 2r - 1, and
 // (cos, sin)(ph) = -(cos, sin)(2 pi r); 1 - tanh^2 = 4 r (1 - r).  Where (1+q)(1+q^2) overflows
 // m = r = 0, where q underflows m = r = 1, and every term stays finite.
+template <bool PLAIN>
 __device__ __forceinline__ float prelude_du(float u, float lr, float li, bool act, float tau)
 {
     float x = u, dxdu = 1.f;
-    if (act) {
+    if (!PLAIN && act) {
         const float v = fminf(fmaxf(u, -50.f), 50.f);
         const float sg = __fdividef(1.f, 1.f + __expf(-v));
         x = v * sg;
@@ -262,12 +263,12 @@ __device__ __forceinline__ float prelude_du(float u, float lr, float li, bool ac
     const float m = p2 * rr, r = p1 * rr;
     float sn, cs;                                    // of 2 pi r: the negated sine and cosine of the phase
     sincos_ftz(r * 6.28318530717959f, sn, cs);
-    const bool open = act || u >= tau;           // with clamp + SiLU every gate is open (see the forward)
+    const bool open = (!PLAIN && act) || u >= tau;           // with clamp + SiLU every gate is open (see the forward)
     const float dm = -fmaf(lr, cs, li * sn);
     const float dph = (open ? m : 0.f) * fmaf(lr, sn, -li * cs);
     // d ph / dx = pi (1 - tanh^2) = 4 pi r (1 - r);  d m / dx = m (1 - m)
     const float dx = fmaf(dm * m, 1.f - m, dph * (12.5663706143592f * r) * (1.f - r));
-    return dx * dxdu;
+    return PLAIN ? dx : dx * dxdu;
 }
 
 // MASKED = false compiles the gate-mask output out (the caller then never passes a mask), which
@@ -611,9 +612,11 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
         // come from one reciprocal of (1+q)(1+q^2).  q is capped at 2^60 so that 1+q^2 stays finite;
         // where the product overflows its reciprocal is +0 and m = r = 0, a q that underflows gives
         // m = r = 1: the right limits.
-        auto push = [&](float u, bool valid, float &zr, float &zi) -> bool {
+        // `plain`: every tap present and no clamp + SiLU, the common case, compiled without the tests
+        auto push = [&](auto plain, float u, bool valid, float &zr, float &zi) -> bool {
+            constexpr bool PLAIN = decltype(plain)::value;
             float x = u;
-            if (act) {
+            if (!PLAIN && act) {
                 x = fminf(fmaxf(x, -50.f), 50.f);
                 x = __fdividef(x, 1.f + __expf(-x));
             }
@@ -625,59 +628,63 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
             sincos_ftz(r * 6.28318530717959f, sn, cs);
             // with clamp + SiLU the magnitude never falls below 0.43, and the host only admits
             // thresholds under that: every gate is open
-            const bool open = valid && (act || u >= tau);
+            const bool open = valid && ((!PLAIN && act) || u >= tau);
             const float mn = open ? -m : 0.f;
             zr = mn * cs; zi = mn * sn;
             return open;
         };
+        auto groups = [&](auto plain) {
+            constexpr bool PLAIN = decltype(plain)::value;
 #pragma unroll
-        for (int gi = 0; gi < NG; ++gi) {
-            // the group's GR new hidden rows come out of the slice together, then the warp
-            // synchronises once: the pushes of these GR steps only reach rows read by now
-            if (gi > 0 && !fused_tail_group) cp_async_wait_pending(NG - 1 - gi);
+            for (int gi = 0; gi < NG; ++gi) {
+                // the group's GR new hidden rows come out of the slice together, then the warp
+                // synchronises once: the pushes of these GR steps only reach rows read by now
+                if (gi > 0 && !fused_tail_group) cp_async_wait_pending(NG - 1 - gi);
 #pragma unroll
-            for (int q = 0; q < GR; ++q) hq[q] = hidden_row(gi * GR + kHalo + q);
-            __syncwarp();
+                for (int q = 0; q < GR; ++q) hq[q] = hidden_row(gi * GR + kHalo + q);
+                __syncwarp();
 #pragma unroll
-            for (int q = 0; q < GR; ++q) {
-                const int i = gi * GR + q;
-                const float2 hv3 = hq[q];
-                float uA = bA, uB = bB;
-                if (tap0) { uA = fmaf(wA[0], hv0.x, uA); uB = fmaf(wB[0], hv0.y, uB); }     // fmaf per channel, tap order
-                if (tap1) { uA = fmaf(wA[1], hv1.x, uA); uB = fmaf(wB[1], hv1.y, uB); }
-                if (tap2) { uA = fmaf(wA[2], hv2.x, uA); uB = fmaf(wB[2], hv2.y, uB); }
-                uA = fmaf(wA[3], hv3.x, uA); uB = fmaf(wB[3], hv3.y, uB);
-                hv0 = hv1; hv1 = hv2; hv2 = hv3;
-                float4 z;
-                const bool oA = push(uA, vA, z.x, z.y), oB = push(uB, vB, z.z, z.w);
-                xs[i * 32] = z;
-                if (want_mask) {
-                    const unsigned bits = ((oA ? 1u : 0u) | (oB ? 2u : 0u)) << (2 * (lane & 15));
-                    const unsigned w0 = __reduce_or_sync(0xffffffffu, lane < 16 ? bits : 0u);
-                    const unsigned w1 = __reduce_or_sync(0xffffffffu, lane < 16 ? 0u : bits);
-                    // rows are parked in lanes and stored sixteen at a time
-                    if (lane == (i & 15)) mkeep = w0;
-                    if (lane == 16 + (i & 15)) mkeep = w1;
-                    if ((i & 15) == 15 || i == T - 1) {
-                        const int r = i - (i & 15) + (lane & 15);
-                        if ((lane & 15) <= (i & 15) && (FULL || r < nvalid) && (lane < 16 || second_word))
-                            mrow0[(long long)r * prm.MW + (lane >> 4)] = mkeep;
+                for (int q = 0; q < GR; ++q) {
+                    const int i = gi * GR + q;
+                    const float2 hv3 = hq[q];
+                    float uA = bA, uB = bB;
+                    if (PLAIN || tap0) { uA = fmaf(wA[0], hv0.x, uA); uB = fmaf(wB[0], hv0.y, uB); }     // fmaf per channel, tap order
+                    if (PLAIN || tap1) { uA = fmaf(wA[1], hv1.x, uA); uB = fmaf(wB[1], hv1.y, uB); }
+                    if (PLAIN || tap2) { uA = fmaf(wA[2], hv2.x, uA); uB = fmaf(wB[2], hv2.y, uB); }
+                    uA = fmaf(wA[3], hv3.x, uA); uB = fmaf(wB[3], hv3.y, uB);
+                    hv0 = hv1; hv1 = hv2; hv2 = hv3;
+                    float4 z;
+                    const bool oA = push(plain, uA, vA, z.x, z.y), oB = push(plain, uB, vB, z.z, z.w);
+                    xs[i * 32] = z;
+                    if (want_mask) {
+                        const unsigned bits = ((oA ? 1u : 0u) | (oB ? 2u : 0u)) << (2 * (lane & 15));
+                        const unsigned w0 = __reduce_or_sync(0xffffffffu, lane < 16 ? bits : 0u);
+                        const unsigned w1 = __reduce_or_sync(0xffffffffu, lane < 16 ? 0u : bits);
+                        // rows are parked in lanes and stored sixteen at a time
+                        if (lane == (i & 15)) mkeep = w0;
+                        if (lane == 16 + (i & 15)) mkeep = w1;
+                        if ((i & 15) == 15 || i == T - 1) {
+                            const int r = i - (i & 15) + (lane & 15);
+                            if ((lane & 15) <= (i & 15) && (FULL || r < nvalid) && (lane < 16 || second_word))
+                                mrow0[(long long)r * prm.MW + (lane >> 4)] = mkeep;
+                        }
                     }
-                }
-                if (FULL || i < nvalid) {
-                    if constexpr (DYN) {
-                        // e <- gamma_t (a e) + z, the factor pair kept for phase 3
-                        const float2 gm = make_float2(vA ? sigmoidf_fast(lgf[i].x + fbA) : 0.f,
-                                                      vB ? sigmoidf_fast(lgf[i].y + fbB) : 0.f);
-                        sm.sG[w * T + i][lane] = gm;
-                        dprod.x *= gm.x; dprod.y *= gm.y;
-                        e = scale_step2(a, e, gm, z);
-                    } else {
-                        e = cfma2(a, e, z);
+                    if (FULL || i < nvalid) {
+                        if constexpr (DYN) {
+                            // e <- gamma_t (a e) + z, the factor pair kept for phase 3
+                            const float2 gm = make_float2(vA ? sigmoidf_fast(lgf[i].x + fbA) : 0.f,
+                                                          vB ? sigmoidf_fast(lgf[i].y + fbB) : 0.f);
+                            sm.sG[w * T + i][lane] = gm;
+                            dprod.x *= gm.x; dprod.y *= gm.y;
+                            e = scale_step2(a, e, gm, z);
+                        } else {
+                            e = cfma2(a, e, z);
+                        }
                     }
                 }
             }
-        }
+        };
+        if (Kc == 4 && !act) groups(std::true_type{}); else groups(std::false_type{});
     } else if constexpr (KIND == KIND_FWD) {
         // |p| >= eps decided as re^2 + im^2 >= eps^2 in double: both squares are exact there
         // and the sum rounds once, so the decision is reproducible bit for bit.  The fp32 sum
@@ -1002,16 +1009,17 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
         }
         // one row of the MIXBWD form: lam -> du, kept in the row's (spent) input slot for the
         // conv transpose that follows the loop
-        auto mix_row = [&](int i, float4 lam) {
+        auto mix_row = [&](auto plain, int i, float4 lam) {
+            constexpr bool PLAIN = decltype(plain)::value;    // every tap present, no clamp + SiLU: no tests
             hwin[0] = hwin[1]; hwin[1] = hwin[2]; hwin[2] = hwin[3];
             hwin[3] = *reinterpret_cast<const float2 *>(&sm.hrev[w * T + i + 3][2 * lane]);
             float uA = mbA, uB = mbB;                    // the forward's fmaf chain, tap order
-            if (mtap0) { uA = fmaf(mwA[0], hwin[3].x, uA); uB = fmaf(mwB[0], hwin[3].y, uB); }
-            if (mtap1) { uA = fmaf(mwA[1], hwin[2].x, uA); uB = fmaf(mwB[1], hwin[2].y, uB); }
-            if (mtap2) { uA = fmaf(mwA[2], hwin[1].x, uA); uB = fmaf(mwB[2], hwin[1].y, uB); }
+            if (PLAIN || mtap0) { uA = fmaf(mwA[0], hwin[3].x, uA); uB = fmaf(mwB[0], hwin[3].y, uB); }
+            if (PLAIN || mtap1) { uA = fmaf(mwA[1], hwin[2].x, uA); uB = fmaf(mwB[1], hwin[2].y, uB); }
+            if (PLAIN || mtap2) { uA = fmaf(mwA[2], hwin[1].x, uA); uB = fmaf(mwB[2], hwin[1].y, uB); }
             uA = fmaf(mwA[3], hwin[0].x, uA); uB = fmaf(mwB[3], hwin[0].y, uB);
-            const float duA = vA ? prelude_du(uA, lam.x, lam.y, mact, prm.gate_tau) : 0.f;
-            const float duB = vB ? prelude_du(uB, lam.z, lam.w, mact, prm.gate_tau) : 0.f;
+            const float duA = vA ? prelude_du<PLAIN>(uA, lam.x, lam.y, mact, prm.gate_tau) : 0.f;
+            const float duB = vB ? prelude_du<PLAIN>(uB, lam.z, lam.w, mact, prm.gate_tau) : 0.f;
             *reinterpret_cast<float2 *>(&xs[i * 32]) = make_float2(duA, duB);
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
@@ -1033,7 +1041,7 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
             }
             dwin[2] = dwin[1]; dwin[1] = dwin[0]; dwin[0] = make_float2(duA, duB);
         };
-        auto step_row = [&](int i, bool clamped) {
+        auto step_row = [&](auto plain, int i, bool clamped) {
             if (MIX && !(FULL || i < nvalid)) *reinterpret_cast<float2 *>(&xs[i * 32]) = make_float2(0.f, 0.f);      // no such row: its du is 0
             if (FULL || i < nvalid) {
                 float2 gown = make_float2(0.f, 0.f);
@@ -1044,7 +1052,7 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
                 } else {
                     P = cfma2(a, P, xs[i * 32]);
                 }
-                if constexpr (MIX) mix_row(i, clamped ? clamp4(P, cl) : P);
+                if constexpr (MIX) mix_row(plain, i, clamped ? clamp4(P, cl) : P);
                 else store_row(i, clamped ? clamp4(P, cl) : P);
                 if constexpr (REV) {
                     // conj(lam) * P_{t-1}
@@ -1085,12 +1093,19 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
                 }
             }
         };
-        if (cl > 0.f) {
+        auto rows = [&](auto plain) {
+            if (cl > 0.f) {
 #pragma unroll
-            for (int i = 0; i < T; ++i) step_row(i, true);
+                for (int i = 0; i < T; ++i) step_row(plain, i, true);
+            } else {
+#pragma unroll
+                for (int i = 0; i < T; ++i) step_row(plain, i, false);
+            }
+        };
+        if constexpr (MIX) {
+            if (prm.conv_k == 4 && !mact) rows(std::true_type{}); else rows(std::false_type{});
         } else {
-#pragma unroll
-            for (int i = 0; i < T; ++i) step_row(i, false);
+            rows(std::false_type{});
         }
         sacc_out = sacc;
         if constexpr (DYN && REV) {
