@@ -90,9 +90,12 @@ enum {
                                                state, state_out and the conv history stay fp32 (the
                                                paper runs a bf16 network around an fp32 scan:
                                                Section "Mixed-Precision and Float32
-                                               Stabilization").  Not available with the time-varying retention,
-                                               the Ear epilogue, the host-staged forward or any
-                                               backward: CAWN_ERR_UNSUPPORTED.                          */
+                                               Stabilization").  With the time-varying retention or the
+                                               Ear epilogue (the paper's own layer form) the two flags
+                                               come together or not at all; the Ear's z_conv is then
+                                               bfloat16 [B, L, 2, H, K].  Not available for the
+                                               host-staged forward or any backward:
+                                               CAWN_ERR_UNSUPPORTED.                                    */
 };
 
 /* Operation selector of cawn_workspace_bytes(). */
@@ -210,9 +213,10 @@ CAWN_API int cawn_phase_accumulate_bwd(const cawn_params *params,
  *   grad_theta_j = sum_{b,t} Re(conj(lam_t) i a_t P_{t-1})      grad_state_in = conj(a_0) lam_0
  * gamma_logit [B,L,H], freq_bias [F] (device).  grad_gamma_logit [B,L,H] float, grad_freq_bias [F]
  * float, grad_theta [C] float: device or NULL.  Other arguments as cawn_phase_accumulate_bwd.
- * grad_gamma_logit is accumulated with atomic adds (zeroed by the call first): when a head spans
- * three or more 64-channel groups (F > 128) its last bits may differ from run to run; everything
- * else is bitwise repeatable.
+ * grad_gamma_logit: where a 64-channel group holds whole heads (F divides 64, or C <= 64) every entry
+ * is the sum of one warp and is stored; otherwise the call zeroes the array and accumulates with
+ * atomic adds, and when a head spans three or more groups (F > 128) its last bits may differ from
+ * run to run.  Everything else is bitwise repeatable.
  */
 CAWN_API int cawn_phase_accumulate_bwd_dynamic(const cawn_params *params,
                                                const void *saved, int saved_kind,
@@ -262,8 +266,8 @@ CAWN_API int cawn_mixing_bwd(const cawn_params *params,
  * CAWN_FLAG_RETENTION_DYNAMIC, which params->flags must carry): the backward of the whole
  * Resonance mixing step as the paper defines it — Temporal Syntax Cache, gated push, per-token
  * per-head retention (Section "Multi-Head Dynamic Parameter Projection").  gamma_logit [B,L,H],
- * freq_bias [F] replace gamma; grad_gamma_logit [B,L,H] (zeroed by the call, then accumulated
- * with atomic adds) and grad_freq_bias [F] replace grad_gamma; each may be NULL.  Everything
+ * freq_bias [F] replace gamma; grad_gamma_logit [B,L,H] (as in cawn_phase_accumulate_bwd_dynamic)
+ * and grad_freq_bias [F] replace grad_gamma; each may be NULL.  Everything
  * else as cawn_mixing_bwd, including the workspace size.
  */
 CAWN_API int cawn_mixing_bwd_dynamic(const cawn_params *params,
@@ -291,6 +295,8 @@ CAWN_API int cawn_mixing_bwd_dynamic(const cawn_params *params,
  * Conv1d layer.  ear_k = 1 with ear_w = 1 and no bias gives the planar Z itself.
  * ear_w:   [2H, ear_k] float (device).  ear_bias: [2H] float (device) or NULL.
  * z_conv:  [B, L, 2, H, K] float (device, 16-byte aligned), K = params->F; as many bytes as y.
+ *          With CAWN_FLAG_INPUT_BF16 | CAWN_FLAG_OUTPUT_BF16 it holds bfloat16 instead (pass the pointer
+ *          as it is).
  * state_out (if given) still receives the unclamped, unconvolved P_{L-1} (and the conv history).
  * Limits: K must divide 64 unless H*K <= 64 (a CTA owns 64 adjacent channels and does not read
  * its neighbours' harmonics).

@@ -162,12 +162,14 @@ inline int io_of(const cawn_params *p)
 
 inline cudaError_t launch_fwd(TileShape ts, const ScanParams &sp, cudaStream_t st, bool dyn = false, int io = 0)
 {
+    if (io != 0 && (dyn || sp.ear_w != nullptr)) return launch_fwd_bf16_wide(ts, sp, st, dyn);
     if (io != 0) return launch_fwd_bf16(ts, sp, st, io);
     if (sp.ear_w != nullptr) return dyn ? launch_fwd_ear_dynamic(ts, sp, st) : launch_fwd_ear(ts, sp, st);
     return dyn ? launch_fwd_dynamic(ts, sp, st) : launch_fwd_static(ts, sp, st);
 }
 inline cudaError_t launch_fused(TileShape ts, const ScanParams &sp, cudaStream_t st, int io = 0, bool dyn = false)
 {
+    if (io != 0 && (dyn || sp.ear_w != nullptr)) return launch_fused_bf16_wide(ts, sp, st, dyn);
     if (dyn) return sp.ear_w != nullptr ? launch_fused_ear_dynamic(ts, sp, st) : launch_fused_dynamic(ts, sp, st);
     if (io != 0) return launch_fused_bf16(ts, sp, st, io);
     return sp.ear_w != nullptr ? launch_fused_ear(ts, sp, st) : launch_fused_plain(ts, sp, st);
@@ -323,7 +325,8 @@ static int fwd_common(const cawn_params *params, const void *input,
     const bool dyn = (params->flags & CAWN_FLAG_RETENTION_DYNAMIC) != 0;
     const bool fused = params->conv_k != 0;
     const int io = io_of(params);
-    if (io != 0 && (dyn || ear_w != nullptr)) return CAWN_ERR_UNSUPPORTED;
+    // with time-varying retention or the Ear epilogue, bf16 storage is built for input and output together
+    if (io != 0 && io != (IO_IN_BF16 | IO_OUT_BF16) && (dyn || ear_w != nullptr)) return CAWN_ERR_UNSUPPORTED;
     if (ear_w != nullptr) {
         if (ear_k != 1 && ear_k != 3) return CAWN_ERR_UNSUPPORTED;
         // a CTA owns 64 adjacent channels: a head's harmonics must not straddle two of them

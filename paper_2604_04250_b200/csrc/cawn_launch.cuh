@@ -20,6 +20,9 @@ cudaError_t launch_fused_dynamic(TileShape ts, const ScanParams &sp, cudaStream_
 // bf16 storage of the input (io & IO_IN_BF16) and / or the output (io & IO_OUT_BF16); io != 0
 cudaError_t launch_fwd_bf16(TileShape ts, const ScanParams &sp, cudaStream_t st, int io);
 cudaError_t launch_fused_bf16(TileShape ts, const ScanParams &sp, cudaStream_t st, int io);
+// bf16 input and output together with time-varying retention (dyn) and / or the Ear epilogue (sp.ear_w)
+cudaError_t launch_fwd_bf16_wide(TileShape ts, const ScanParams &sp, cudaStream_t st, bool dyn);
+cudaError_t launch_fused_bf16_wide(TileShape ts, const ScanParams &sp, cudaStream_t st, bool dyn);
 cudaError_t launch_bwd_static(TileShape ts, const ScanParams &sp, cudaStream_t st);    // reverse scan
 cudaError_t launch_bwd_dynamic(TileShape ts, const ScanParams &sp, cudaStream_t st);
 cudaError_t launch_mix_bwd(TileShape ts, const ScanParams &sp, cudaStream_t st);       // reverse scan + prelude backward

@@ -278,7 +278,7 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
                                           const int g, const int b, const int k)
 {
     static_assert(!(EAR && kind_is_bwd(KIND)), "the Ear epilogue belongs to the forward");
-    static_assert(IO == IO_F32 || (!EAR && !DYN && !kind_is_bwd(KIND)), "bf16 storage is built for the static forward");
+    static_assert(IO == IO_F32 || !kind_is_bwd(KIND), "bf16 storage is built for the forward");
     constexpr bool IN16 = (IO & IO_IN_BF16) != 0, OUT16 = (IO & IO_OUT_BF16) != 0;
     constexpr bool REV = kind_is_bwd(KIND);
     constexpr bool MIX = (KIND == KIND_MIXBWD);
@@ -919,7 +919,9 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
 
         // EAR: a planar row is 2C floats, as long as an interleaved one; the real parts of this
         // lane's two channels sit c0 floats into it, the imaginary parts C floats further
-        char *const rbase = reinterpret_cast<char *>(prm.out) + (EAR ? (e0 - c0) * 8 + c0 * 4 : (OUT16 ? e0 * 4 : e0 * 8));
+        // (with bf16 output every one of these offsets halves)
+        char *const rbase = reinterpret_cast<char *>(prm.out) +
+                            (EAR ? ((e0 - c0) * 8 + c0 * 4) / (OUT16 ? 2 : 1) : (OUT16 ? e0 * 4 : e0 * 8));
         const int orow = OUT16 ? rowbytes / 2 : rowbytes;
         const float cl = prm.clampv;
         // Ear taps of this lane's two channels, real and imaginary part: (left, centre, right,
@@ -949,7 +951,7 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
         // form exchanges edge channels with the neighbouring lanes)
         auto store_row = [&](int i, float4 o) {
             char *r = const_cast<char *>(row_ptr(rbase, orow, i));
-            if constexpr (OUT16) {
+            if constexpr (OUT16 && !EAR) {
                 const unsigned pA = float2_to_bf16x2(o.x, o.y), pB = float2_to_bf16x2(o.z, o.w);
                 if (VEC) {
                     if (vA) __stcs(reinterpret_cast<uint2 *>(r), make_uint2(pA, pB));
@@ -964,12 +966,24 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
                 const float zrB = fmaf(ewr[1][0], o.x, fmaf(ewr[1][1], o.z, fmaf(ewr[1][2], rre, ewr[1][3])));
                 const float ziA = fmaf(ewi[0][0], lim, fmaf(ewi[0][1], o.y, fmaf(ewi[0][2], o.w, ewi[0][3])));
                 const float ziB = fmaf(ewi[1][0], o.y, fmaf(ewi[1][1], o.w, fmaf(ewi[1][2], rim, ewi[1][3])));
-                float *zr = reinterpret_cast<float *>(r), *zi = zr + C;
-                if (VEC) {
-                    if (vA) { __stcs(reinterpret_cast<float2 *>(zr), make_float2(zrA, zrB)); __stcs(reinterpret_cast<float2 *>(zi), make_float2(ziA, ziB)); }
+                if constexpr (OUT16) {
+                    // planar row of 2C bf16: real parts, then imaginary parts
+                    unsigned short *zr = reinterpret_cast<unsigned short *>(r), *zi = zr + C;
+                    const unsigned pr = float2_to_bf16x2(zrA, zrB), pi = float2_to_bf16x2(ziA, ziB);
+                    if (VEC) {
+                        if (vA) { __stcs(reinterpret_cast<unsigned *>(zr), pr); __stcs(reinterpret_cast<unsigned *>(zi), pi); }
+                    } else {
+                        if (vA) { zr[0] = (unsigned short)(pr & 0xffffu); zi[0] = (unsigned short)(pi & 0xffffu); }
+                        if (vB) { zr[1] = (unsigned short)(pr >> 16); zi[1] = (unsigned short)(pi >> 16); }
+                    }
                 } else {
-                    if (vA) { __stcs(zr, zrA); __stcs(zi, ziA); }
-                    if (vB) { __stcs(zr + 1, zrB); __stcs(zi + 1, ziB); }
+                    float *zr = reinterpret_cast<float *>(r), *zi = zr + C;
+                    if (VEC) {
+                        if (vA) { __stcs(reinterpret_cast<float2 *>(zr), make_float2(zrA, zrB)); __stcs(reinterpret_cast<float2 *>(zi), make_float2(ziA, ziB)); }
+                    } else {
+                        if (vA) { __stcs(zr, zrA); __stcs(zi, ziA); }
+                        if (vB) { __stcs(zr + 1, zrB); __stcs(zi + 1, ziB); }
+                    }
                 }
             } else if (VEC) {
                 // 16-byte rows go out as st.global.cg (kept in L2 until evicted: measured 0.5 us faster on

@@ -107,9 +107,78 @@ def test_fused_bf16_storage(B, L, C, Kc, in16, out16):
     assert np.array_equal(unpack_mask(m.cpu().numpy().view(np.uint32), C), rmask)
 
 
+@pytest.mark.parametrize("fused", [False, True])
+@pytest.mark.parametrize("dyn,ear", [(True, False), (False, True), (True, True)])
+@pytest.mark.parametrize("B,L,H,F", [(1, 2, 1, 64), (2, 200, 2, 64), (1, 333, 4, 16), (2, 515, 12, 64), (1, 131, 3, 11)])
+def test_bf16_with_dynamic_retention_and_ear(B, L, H, F, dyn, ear, fused):
+    """bf16 input and output around the fp32 scan in the forms of the paper's own layer: per-token
+    retention and / or the Ear's convolution across the harmonics as the epilogue, Cartesian and
+    fused input.  The oracle gets the widened bf16 inputs; the bf16 output is compared within its
+    own rounding."""
+    import torch
+    from gpu_util import dev, state_blob, split_blob
+    from paper_2604_04250_b200 import binding as cb
+    C = H * F
+    if ear and C > 64 and 64 % F != 0:
+        pytest.skip("the Ear epilogue needs the harmonics of a head inside one 64-channel group")
+    eps, tau, Kc = 0.1, float(inputs.gate_tau(0.1)), 4
+    rng = np.random.default_rng(1000 + L + F)
+    P_in = (rng.normal(0, 2, (B, C)) + 1j * rng.normal(0, 2, (B, C))).astype(np.complex64)
+    dd = inputs.dynamic_retention_inputs(B, L, H, F, 1100 + L) if dyn else {}
+    ew = rng.normal(0.0, 0.6, (2 * H, 3)).astype(np.float32)
+    eb = rng.normal(0.0, 0.3, 2 * H).astype(np.float32)
+    flags = _io_flags(cb, True, True) | (cb.CAWN_FLAG_RETENTION_DYNAMIC if dyn else 0)
+    kw = dict(gamma_logit=dev(dd.get("gamma_logit")), freq_bias=dev(dd.get("freq_bias")))
+    okw = dict(gamma_logit=dd.get("gamma_logit"), freq_bias=dd.get("freq_bias"), H=H) if dyn else {}
+    if fused:
+        d = inputs.fused_inputs(B, L, C, 1200 + L, conv_k=Kc, with_tail=True, with_bias=True)
+        bits, wide = inputs.to_bf16(d["h"])
+        y_ref, so_ref, m_ref, tail_ref = oracle.fused_forward(wide, d["conv_w"], None if dyn else d["gamma"], d["theta"], eps, tau,
+                                                              bias=d["conv_bias"], tail_in=d["tail_in"],
+                                                              state_in=P_in.astype(np.complex128), **okw)
+        prm = cb.make_params(B, L, H, F, gate_eps=eps, gate_tau=tau, conv_k=Kc, flags=flags)
+        s_in, off = state_blob(B, C, Kc, P_in, d["tail_in"])
+        s_out, _ = state_blob(B, C, Kc)
+        kw.update(conv_w=dev(d["conv_w"]), conv_bias=dev(d["conv_bias"]))
+    else:
+        d = inputs.scan_inputs(B, L, C, 1200 + L)
+        bits, wide = inputs.to_bf16(d["p"])
+        z, m_ref = oracle.gate(wide, eps)
+        y_ref, so_ref = oracle.scan(z, d["theta"], gamma=None if dyn else d["gamma"], state_in=P_in.astype(np.complex128), **okw)
+        prm = cb.make_params(B, L, H, F, gate_eps=eps, flags=flags)
+        s_in = dev(P_in)
+        s_out = torch.full((B, C), float("nan"), dtype=torch.complex64, device="cuda")
+    ws = cb.new_workspace(prm, cb.CAWN_OP_FWD)
+    x = torch.from_numpy(bits.view(np.int16)).cuda()
+    m = torch.zeros((B, L, (C + 31) // 32), dtype=torch.int32, device="cuda")
+    g = None if dyn else dev(d["gamma"])
+    if ear:
+        zc = torch.full((B, L, 2, H, F), -1, dtype=torch.int16, device="cuda")
+        cb.cawn_phase_accumulate_fwd_ear(prm, x, g, dev(d["theta"]), dev(ew), 3, zc, ws, ear_bias=dev(eb), state_in=s_in,
+                                         state_out=s_out, gate_mask=m, **kw)
+        got = inputs.from_bf16(zc.cpu().numpy().view(np.uint16))
+        want = oracle.ear_conv(y_ref, ew, eb, H, F)
+    else:
+        y = torch.full((B, L, C, 2), -1, dtype=torch.int16, device="cuda")
+        cb.cawn_phase_accumulate_fwd(prm, x, g, dev(d["theta"]), y, ws, state_in=s_in, state_out=s_out, gate_mask=m, **kw)
+        got = _read_y(y, True)
+        want = y_ref
+    assert cb.cawn_poll_status(ws) == 0
+    assert not np.isnan(got.view(np.float32)).any()
+    assert floored_rel_err(got, want) < TOL16
+    if fused:
+        P_out, tail_out = split_blob(s_out, off, B, C, Kc)
+        assert np.array_equal(tail_out, tail_ref.astype(np.float32))
+    else:
+        P_out = s_out.cpu().numpy()
+    assert floored_rel_err(P_out, so_ref) < TOL                      # the carried state stays fp32
+    assert np.array_equal(unpack_mask(m.cpu().numpy().view(np.uint32), C), m_ref)
+
+
 def test_bf16_refused_where_not_built():
     import torch
     from paper_2604_04250_b200 import binding as cb
+    # with the Ear epilogue (or time-varying retention) bf16 storage comes for input and output together
     prm = cb.make_params(1, 8, 1, 64, flags=cb.CAWN_FLAG_OUTPUT_BF16)
     ws = cb.new_workspace(prm, cb.CAWN_OP_FWD)
     x = torch.zeros((1, 8, 64), dtype=torch.complex64, device="cuda")
