@@ -7,7 +7,7 @@ namespace cawn {
 // The float4 path needs every row segment on a 16-byte boundary: C even (the arrays
 // themselves are checked to be 16-byte aligned).  The tile is staged in dynamic shared memory;
 // MINB is the number of CTAs per SM the register allocation leaves room for.
-template <int T, int W, int KIND, bool VEC, int MINB, bool DYN, bool EAR = false, int IO = IO_F32, bool MASKED = true>
+template <int T, int W, int KIND, bool VEC, int MINB, bool DYN, bool EAR = false, int IO = IO_F32, bool MASKED = true, bool LATE = false>
 cudaError_t launch_scan_inst(const ScanParams &sp, cudaStream_t st)
 {
     constexpr size_t smem = sizeof(ScanSmem<T, W, KIND, DYN>);
@@ -16,7 +16,7 @@ cudaError_t launch_scan_inst(const ScanParams &sp, cudaStream_t st)
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= 64 || !configured[dev]) {
-        e = cudaFuncSetAttribute(cawn_scan_kernel<T, W, KIND, VEC, MINB, DYN, EAR, IO, MASKED>,
+        e = cudaFuncSetAttribute(cawn_scan_kernel<T, W, KIND, VEC, MINB, DYN, EAR, IO, MASKED, LATE>,
                                  cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) configured[dev] = true;
@@ -34,13 +34,13 @@ cudaError_t launch_scan_inst(const ScanParams &sp, cudaStream_t st)
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, cawn_scan_kernel<T, W, KIND, VEC, MINB, DYN, EAR, IO, MASKED>, sp);
+    return cudaLaunchKernelEx(&cfg, cawn_scan_kernel<T, W, KIND, VEC, MINB, DYN, EAR, IO, MASKED, LATE>, sp);
 }
-template <int T, int W, int KIND, int MINB, bool DYN = false, bool EAR = false, int IO = IO_F32, bool MASKED = true>
+template <int T, int W, int KIND, int MINB, bool DYN = false, bool EAR = false, int IO = IO_F32, bool MASKED = true, bool LATE = false>
 cudaError_t launch_scan(const ScanParams &sp, cudaStream_t st)
 {
-    return sp.C % 2 == 0 ? launch_scan_inst<T, W, KIND, true, MINB, DYN, EAR, IO, MASKED>(sp, st)
-                         : launch_scan_inst<T, W, KIND, false, MINB, DYN, EAR, IO, MASKED>(sp, st);
+    return sp.C % 2 == 0 ? launch_scan_inst<T, W, KIND, true, MINB, DYN, EAR, IO, MASKED, LATE>(sp, st)
+                         : launch_scan_inst<T, W, KIND, false, MINB, DYN, EAR, IO, MASKED, LATE>(sp, st);
 }
 // The bf16 storage forms of the static forward (io = IO_IN_BF16, IO_OUT_BF16 or both).
 template <int KIND, int IO>

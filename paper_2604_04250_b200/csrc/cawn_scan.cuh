@@ -144,6 +144,7 @@ struct ScanSmem {
     float2 sRD[DYN ? kWindow + 1 : 1][DYN ? 32 : 1];  // DYN: factor products of the window's tiles
     float2 sG[DYN ? TILE : 1][DYN ? 32 : 1];          // DYN: each row's own factor pair, kept from phase 1 for phase 3
     unsigned long long epoch;
+    unsigned arrived;                                  // thread 0: this CTA's arrival count
     int err;
     unsigned hook;                                     // copy of the workspace's wait hook
 };
@@ -273,7 +274,7 @@ __device__ __forceinline__ float prelude_du(float u, float lr, float li, bool ac
 
 // MASKED = false compiles the gate-mask output out (the caller then never passes a mask), which
 // keeps its registers out of the plain forward.
-template <int T, int W, int KIND, bool VEC, bool DYN, bool FULL, bool EAR = false, int IO = IO_F32, bool MASKED = true>
+template <int T, int W, int KIND, bool VEC, bool DYN, bool FULL, bool EAR = false, int IO = IO_F32, bool MASKED = true, bool LATE = false>
 __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, KIND, DYN> &sm,
                                           const int g, const int b, const int k)
 {
@@ -321,6 +322,11 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
         }
     }
     const bool early = !REV && prm.early_loads != 0;
+    // LATE (static Cartesian forward without a mask, a call whose CTAs are all resident at once, the
+    // input vouched for): the gate pass, which reads the input rows and writes shared memory only,
+    // runs before the wait for the previous launch.
+    static_assert(!LATE || (KIND == KIND_FWD && !DYN && !MASKED), "the late wait is built for the plain forward");
+    const bool late_wait = LATE && early;
     if (!early) grid_wait_previous();
     // Fused path: every warp stages its own T hidden rows (floats) behind kHalo rows of history in
     // the upper part of its own T x 512-byte slice of the tile, row r at byte 256 (T - 3) + 256 r
@@ -483,17 +489,20 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
         o[0] = (float)c1r; o[1] = (float)c1i; o[2] = (float)cTr; o[3] = (float)cTi; o[4] = (float)cAr; o[5] = (float)cAi;
     }
     // everything below touches what the previous launch may have written (workspace, states)
-    if (early && KIND != KIND_FUSED) grid_wait_previous();
+    if (early && KIND != KIND_FUSED && !late_wait) grid_wait_previous();
     unsigned long long epoch0 = 0;
     unsigned arrived = 0;
-    if (tid == 0) {
+    auto read_epoch = [&]() {                            // thread 0 only
         unsigned hook0;
         ld_epoch_hook(prm.ws, epoch0, hook0);
         sm.epoch = epoch0;
-        sm.err = 0;
         sm.hook = hook0;
         // counted only once the epoch has been read (the increment depends on its value)
         arrived = atomicAdd(&prm.ws->done, 1u + (unsigned)(epoch0 >> 63));
+    };
+    if (tid == 0) {
+        sm.err = 0;
+        if (!late_wait) read_epoch();
     }
     __syncthreads();                                                           // barrier 1
     float4 a, aT;
@@ -504,7 +513,6 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
         a = make_float4(u0.x, u0.y, u1.z, u1.w);
         aT = make_float4(u0.z, u0.w, u2.x, u2.y);
     }
-    const unsigned long long epoch = sm.epoch;
 
     // Time-varying retention: this lane's heads and per-harmonic biases, and the factor pair of
     // one physical row t (0 outside the call, which only ever multiplies a zero carry).
@@ -540,11 +548,14 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
     // The call's initial state is read before this tile publishes anything, so that state_out
     // may alias state_in: whoever writes state_out has waited for every tile's aggregate.
     float4 sinit = zero4();
-    if (!REV && cpt == 0 && w == M % W && prm.state_in != nullptr) {
-        const float2 *sp = prm.state_in + (long long)b * C + c0;
-        if (vA) { const float2 v = sp[0]; sinit.x = v.x; sinit.y = v.y; }
-        if (vB) { const float2 v = sp[1]; sinit.z = v.x; sinit.w = v.y; }
-    }
+    auto read_state_in = [&]() {
+        if (!REV && cpt == 0 && w == M % W && prm.state_in != nullptr) {
+            const float2 *sp = prm.state_in + (long long)b * C + c0;
+            if (vA) { const float2 v = sp[0]; sinit.x = v.x; sinit.y = v.y; }
+            if (vB) { const float2 v = sp[1]; sinit.z = v.x; sinit.w = v.y; }
+        }
+    };
+    if (!late_wait) read_state_in();
 
     if constexpr (REV) {
         cp_async_wait_all();
@@ -720,7 +731,7 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
             for (int i = 0; i < T; ++i) {
                 if (!EXACT && i % GR == 0) {
                     cp_async_wait_pending(NG - 1 - i / GR);       // rows i .. i+GR-1 have landed
-                    if (i == 0 && early_ptr != nullptr) {
+                    if (i == 0 && early_ptr != nullptr && !late_wait) {
                         er0 = ld_record(early_ptr + 2 * lane);
                         er1 = ld_record(early_ptr + 2 * lane + 1);
                     }
@@ -833,12 +844,14 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
     }
     sm.sE[w][lane] = e;
     if constexpr (DYN) sm.sD[w][lane] = dprod;
-    if (tid == 0 && arrived == gridDim.x * gridDim.y * gridDim.z - 1) {
-        // every CTA of this launch has read the epoch: open the next one
-        st_volatile_u32(&prm.ws->done, 0u);
-        st_volatile_u64(&prm.ws->epoch, epoch0 + 1ull);
+    if (late_wait) {
+        // from here on the workspace, the carried state and the outputs are touched
+        grid_wait_previous();
+        if (tid == 0) read_epoch();
+        read_state_in();
     }
     __syncthreads();                                                           // barrier 2
+    const unsigned long long epoch = sm.epoch;
 
     // ---- 2. publish the aggregate, fetch the carry window ----------------------------------
     const unsigned hook = sm.hook;
@@ -889,6 +902,7 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
         }
     }
     __syncthreads();                                                           // barrier 3
+    if (tid == 0) sm.arrived = arrived;              // (it has come back by now) wanted again at the very end
 
     // ---- 3. carry-in, the recurrence itself, stores -----------------------------------------
     const bool failed = (sm.err != 0);
@@ -1280,9 +1294,15 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
             }
         }
     }
+    if (tid == 0 && sm.arrived == gridDim.x * gridDim.y * gridDim.z - 1) {
+        // every CTA of this launch has read the epoch: open the next one (the launch after this
+        // one reads it only when this one is complete)
+        st_volatile_u32(&prm.ws->done, 0u);
+        st_volatile_u64(&prm.ws->epoch, sm.epoch + 1ull);
+    }
 }
 
-template <int T, int W, int KIND, bool VEC, int MINB, bool DYN = false, bool EAR = false, int IO = IO_F32, bool MASKED = true>
+template <int T, int W, int KIND, bool VEC, int MINB, bool DYN = false, bool EAR = false, int IO = IO_F32, bool MASKED = true, bool LATE = false>
 __global__ void __launch_bounds__(W * 32, MINB) cawn_scan_kernel(const ScanParams prm)
 {
     constexpr int TILE = T * W;
@@ -1295,8 +1315,8 @@ __global__ void __launch_bounds__(W * 32, MINB) cawn_scan_kernel(const ScanParam
     const int k = blockIdx.z;                         // tile index along (logical) time
     grid_launch_dependents();
     const bool full = ((long long)(k + 1) * TILE <= prm.L) && (g * 64 + 64 <= prm.C);
-    if (full) scan_tile<T, W, KIND, VEC, DYN, true, EAR, IO, MASKED>(prm, sm, g, b, k);
-    else      scan_tile<T, W, KIND, VEC, DYN, false, EAR, IO, MASKED>(prm, sm, g, b, k);
+    if (full) scan_tile<T, W, KIND, VEC, DYN, true, EAR, IO, MASKED, LATE>(prm, sm, g, b, k);
+    else      scan_tile<T, W, KIND, VEC, DYN, false, EAR, IO, MASKED, LATE>(prm, sm, g, b, k);
 }
 
 }  // namespace cawn
