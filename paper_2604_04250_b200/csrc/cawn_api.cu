@@ -142,8 +142,16 @@ cudaError_t launch_epilogue(EpilogueParams ep, bool want_q, bool want_s, bool wa
     const long long blocks = (long long)ep.nb_q + ep.nb_s + ep.nb_c + seams;
     if (blocks == 0) return cudaSuccess;
     if (blocks > 2147483647ll) return cudaErrorInvalidValue;
-    cawn_bwd_epilogue_kernel<<<(unsigned)blocks, kEpiWarps * 32, 0, st>>>(ep);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)blocks, 1, 1);
+    cfg.blockDim = dim3(kEpiWarps * 32, 1, 1);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, cawn_bwd_epilogue_kernel, ep);
 }
 
 // The logit gradient of a (row, head) is complete inside one 64-channel group when the group holds

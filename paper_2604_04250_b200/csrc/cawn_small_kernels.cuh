@@ -79,13 +79,22 @@ __device__ __forceinline__ void seam_rows(const EpilogueParams &ep, int c, int k
     float wt[4];
 #pragma unroll
     for (int j = 0; j < 4; ++j) wt[j] = j >= 4 - Kc ? ep.conv_w[(long long)c * Kc + (j - (4 - Kc))] : 0.f;
-    // du at physical row r, from whichever tile end holds it
-    auto DU = [&](long long r) -> float {
+    // du at physical row r, from whichever tile end holds it.  r lies within three rows of tile
+    // `base` (the tile whose seam is being finished; for the history rows the last tile), so it
+    // belongs to that tile or to one of its neighbours: no division is needed to find it.
+    auto DU = [&](long long r, int base) -> float {
         if (r < 0 || r >= L) return 0.f;
-        const long long kk = (L - 1 - r) / tile;
-        const long long t_hi = L - 1 - kk * tile;
-        long long t_lo = L - (kk + 1) * tile;
+        long long t_hi = L - 1 - (long long)base * tile;
+        long long t_lo = L - (long long)(base + 1) * tile;
         if (t_lo < 0) t_lo = 0;
+        int kk = base;
+        if (r > t_hi) kk = base - 1; else if (r < t_lo) kk = base + 1;
+        if (kk != base) {
+            t_hi = L - 1 - (long long)kk * tile;
+            t_lo = L - (long long)(kk + 1) * tile;
+            if (t_lo < 0) t_lo = 0;
+        }
+        if (kk < 0 || kk >= K || r > t_hi || r < t_lo) return 0.f;      // never: three rows reach no further
         const float *e = ep.edge_du + (((long long)b * K + kk) * 6) * C + c;
         if (t_hi - r < 3) return e[(t_hi - r) * C];
         if (r - t_lo < 3) return e[(3 + (r - t_lo)) * C];
@@ -98,7 +107,7 @@ __device__ __forceinline__ void seam_rows(const EpilogueParams &ep, int c, int k
         for (long long s = t_hi; s >= t_lo && s > t_hi - 3; --s) {
             float acc = 0.f;
 #pragma unroll
-            for (int j = 0; j < 4; ++j) acc = fmaf(wt[j], DU(s + 3 - j), acc);
+            for (int j = 0; j < 4; ++j) acc = fmaf(wt[j], DU(s + 3 - j, kb), acc);
             if (ep.dtail_out != nullptr && s >= L - Kh) acc += ep.dtail_out[((long long)b * Kh + (s - (L - Kh))) * C + c];
             ep.grad_h[((long long)b * L + s) * C + c] = acc;
         }
@@ -107,7 +116,7 @@ __device__ __forceinline__ void seam_rows(const EpilogueParams &ep, int c, int k
             const long long s = r - Kh;
             float acc = 0.f;
 #pragma unroll
-            for (int j = 0; j < 4; ++j) acc = fmaf(wt[j], DU(s + 3 - j), acc);
+            for (int j = 0; j < 4; ++j) acc = fmaf(wt[j], DU(s + 3 - j, K - 1), acc);
             if (ep.dtail_out != nullptr && r >= L) acc += ep.dtail_out[((long long)b * Kh + (r - L)) * C + c];
             ep.dtail_in[((long long)b * Kh + r) * C + c] = acc;
         }
@@ -117,6 +126,10 @@ __device__ __forceinline__ void seam_rows(const EpilogueParams &ep, int c, int k
 __global__ void __launch_bounds__(kEpiWarps * 32) cawn_bwd_epilogue_kernel(const EpilogueParams ep)
 {
     __shared__ double sh[kEpiWarps * 5 * 32];
+    // launched with programmatic stream serialisation behind the reverse scan: let the launch after
+    // this one start filling SMs, and touch nothing before the scan is complete
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     int blk = blockIdx.x;
     const int C = ep.C, nparts = ep.nparts;
