@@ -101,15 +101,33 @@ __device__ __forceinline__ void seam_rows(const EpilogueParams &ep, int c, int k
         return 0.f;                                  // not an edge row: never asked for
     };
     if (kb < K) {
+        // The three latest rows of tile kb, t_hi - i (i = 0, 1, 2), reach du of rows t_hi + 3 .. t_hi - 2:
+        // the three earliest rows of the tile after it in time (tile kb - 1, its second edge triple)
+        // and this tile's own three latest (its first edge triple; rows it does not have hold 0).
         const long long t_hi = L - 1 - (long long)kb * tile;
         long long t_lo = L - (long long)(kb + 1) * tile;
         if (t_lo < 0) t_lo = 0;
-        for (long long s = t_hi; s >= t_lo && s > t_hi - 3; --s) {
-            float acc = 0.f;
+        const float *own = ep.edge_du + (((long long)b * K + kb) * 6) * C + c;
+        float d[6];                                  // d[m + 2] = du(t_hi + m), m = -2 .. 3
 #pragma unroll
-            for (int j = 0; j < 4; ++j) acc = fmaf(wt[j], DU(s + 3 - j, kb), acc);
-            if (ep.dtail_out != nullptr && s >= L - Kh) acc += ep.dtail_out[((long long)b * Kh + (s - (L - Kh))) * C + c];
-            ep.grad_h[((long long)b * L + s) * C + c] = acc;
+        for (int i = 0; i < 3; ++i) d[2 - i] = own[(long long)i * C];
+        if (kb > 0) {
+            const float *nxt = ep.edge_du + (((long long)b * K + (kb - 1)) * 6 + 3) * C + c;
+#pragma unroll
+            for (int i = 0; i < 3; ++i) d[3 + i] = nxt[(long long)i * C];
+        } else {
+            d[3] = d[4] = d[5] = 0.f;
+        }
+#pragma unroll
+        for (int i = 0; i < 3; ++i) {
+            const long long srow = t_hi - i;
+            if (srow >= t_lo) {
+                float acc = 0.f;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc = fmaf(wt[j], d[(3 - i - j) + 2], acc);
+                if (ep.dtail_out != nullptr && srow >= L - Kh) acc += ep.dtail_out[((long long)b * Kh + (srow - (L - Kh))) * C + c];
+                ep.grad_h[((long long)b * L + srow) * C + c] = acc;
+            }
         }
     } else if (ep.dtail_in != nullptr) {
         for (int r = 0; r < Kh; ++r) {
