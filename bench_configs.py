@@ -217,6 +217,8 @@ def _dev(a):
 def cfg1_variants(cb, inputs, want, seconds):
     import torch
     out = []
+    if not any(want(x) for x in ("plain", "mask", "ear", "bf16", "dynamic")):
+        return out
     cfg = inputs.CONFIGS[1]
     B, L, C = cfg.B, cfg.L, cfg.C
     small = inputs.scan_inputs(1, 1, C, cfg.seed, cfg.gamma_lo, cfg.gamma_hi)
@@ -271,6 +273,8 @@ def cfg1_variants(cb, inputs, want, seconds):
 def cfg2_prefill(cb, inputs, want, seconds):
     import torch
     out = []
+    if not want("cfg2"):
+        return out
     cfg = inputs.CONFIGS[2]
     C, n = cfg.C, cfg.chunk
     small = inputs.scan_inputs(1, 1, C, cfg.seed, cfg.gamma_lo, cfg.gamma_hi)
@@ -310,6 +314,8 @@ def cfg2_prefill(cb, inputs, want, seconds):
 def cfg3_backward(cb, inputs, want, seconds):
     import torch
     out = []
+    if not (want("cfg3") or want("cfg3dyn")):
+        return out
     cfg = inputs.CONFIGS[3]
     B, L, C = cfg.B, cfg.L, cfg.C
     small = inputs.scan_inputs(1, 1, C, cfg.seed, cfg.gamma_lo, cfg.gamma_hi)
@@ -351,6 +357,8 @@ def cfg3_backward(cb, inputs, want, seconds):
 def cfg4_fused(cb, inputs, want, seconds, batch=0):
     import torch
     out = []
+    if not any(want(x) for x in ("cfg4", "cfg4dyn", "cfg4bf16", "cfg4bwd", "cfg4bwddyn")):
+        return out
     cfg = inputs.CONFIGS[4]
     B, L, C = (batch or cfg.B), cfg.L, cfg.C
     tag = "" if B == cfg.B else "_B%d" % B
