@@ -8,7 +8,7 @@
 // is what lets three 64 KB tiles per SM stay in flight next to the arithmetic.
 //
 //   0. every thread issues the asynchronous copies of its own T row pieces, in groups of a few
-//      rows; meanwhile 192 threads prepare the per-channel coefficients a, a^T, a^TILE in
+//      rows; meanwhile 64 threads prepare the per-channel coefficients a, a^T, a^TILE in
 //      double                                                                    [barrier 1]
 //   1. as its row groups land: gate (Cartesian forward; the gated value goes back to shared
 //      memory), and each thread reduces its T steps from a zero start, leaving the end state
