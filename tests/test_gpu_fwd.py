@@ -273,3 +273,29 @@ def test_overlapped_calls_match_serial_calls_bitwise():
     y_ref, so_ref, _ = oracle.forward(p_all, ds[0]["gamma"], ds[0]["theta"], 0.1)
     assert floored_rel_err(np.concatenate(list(outs[1][0]), axis=1), y_ref, axes=(0, 1)) < TOL
     assert floored_rel_err(outs[1][1], so_ref) < TOL
+
+
+def test_config1_as_benched_rotating_buffers():
+    """Config 1 in the launch configuration bench.py times: the input vouched for, no mask, state out,
+    steps issued back to back over rotating buffer sets with no synchronisation in between.  Every
+    step's output against the oracle (the sets are time-rolled copies of one draw, as in the bench)."""
+    import torch
+    from gpu_util import dev
+    from paper_2604_04250_b200 import binding as cb
+    cfg = inputs.CONFIGS[1]
+    d = inputs.config_inputs(cfg)
+    B, L, C, nsets, nsteps = cfg.B, cfg.L, cfg.C, 3, 7
+    p0 = dev(d["p"])
+    ps = [torch.roll(p0, shifts=17 * i, dims=1).contiguous() for i in range(nsets)]
+    ys = [torch.full_like(p0, float("nan")) for _ in range(nsteps)]
+    g, t = dev(d["gamma"]), dev(d["theta"])
+    prm = cb.make_params(B, L, cfg.H, cfg.F, gate_eps=cfg.gate_eps, flags=cb.CAWN_FLAG_INPUT_INDEPENDENT)
+    ws = cb.new_workspace(prm, cb.CAWN_OP_FWD)
+    state = torch.empty((B, C), dtype=torch.complex64, device="cuda")
+    for i in range(nsteps):
+        cb.cawn_phase_accumulate_fwd(prm, ps[i % nsets], g, t, ys[i], ws, state_out=state)
+    assert cb.cawn_poll_status(ws) == 0
+    refs = [oracle.forward(np.roll(d["p"], 17 * i, axis=1), d["gamma"], d["theta"], cfg.gate_eps) for i in range(nsets)]
+    for i in range(nsteps):
+        assert floored_rel_err(ys[i].cpu().numpy(), refs[i % nsets][0], axes=(0, 1)) < TOL, i
+    assert floored_rel_err(state.cpu().numpy(), refs[(nsteps - 1) % nsets][1]) < TOL
