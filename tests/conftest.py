@@ -38,7 +38,8 @@ def built_libraries():
 def pytest_terminal_summary(terminalreporter, exitstatus, config):
     """Parity margins of the run: for every test function that compared something, the largest
     floored error it saw (the quantity the tolerances bound) and the largest unfloored median of
-    the element-wise relative error.  Also written to gpurun_out/parity_margins.json."""
+    the element-wise relative error.  Also written as parity_margins.json into the directory the
+    environment variable CAWN_REPORT_DIR names, when it is set."""
     import json
     try:
         from helpers import MARGINS
@@ -55,7 +56,9 @@ def pytest_terminal_summary(terminalreporter, exitstatus, config):
     for name in sorted(rows):
         n, e, m = rows[name]
         terminalreporter.write_line("%-96s %.3e  %.3e  %d" % (name, e, m, n))
-    out = os.path.join(ROOT, "gpurun_out")
+    out = os.environ.get("CAWN_REPORT_DIR")
+    if not out:
+        return
     try:
         os.makedirs(out, exist_ok=True)
         with open(os.path.join(out, "parity_margins.json"), "w") as f:
