@@ -140,6 +140,22 @@ __device__ __forceinline__ bool poll_pair(const uint4 *tile_recs, int lane, unsi
     }
 }
 
+// Gate-mask words from per-lane bits.  Lane l of a half-warp holds in bit pair i of `m` the two gate
+// bits (its two channels) of row i, i < 16.  Returns, in lane r of the same half-warp, the word
+// whose bit pair l holds what lane l had for row r: the mask word of row r for the half-warp's 32
+// channels.  A 16 x 16 transpose of 2-bit entries over 16 lanes: four butterfly exchanges.
+__device__ __forceinline__ unsigned transpose_pairs16(unsigned m, int lane)
+{
+#pragma unroll
+    for (int d = 8; d >= 1; d >>= 1) {
+        // the bit pairs whose index has bit d clear
+        const unsigned m0 = d == 8 ? 0x0000ffffu : d == 4 ? 0x00ff00ffu : d == 2 ? 0x0f0f0f0fu : 0x33333333u;
+        const unsigned y = __shfl_xor_sync(0xffffffffu, m, d);
+        m = (lane & d) ? ((m & ~m0) | ((y & ~m0) >> (2 * d))) : ((m & m0) | ((y & m0) << (2 * d)));
+    }
+    return m;
+}
+
 // ---------------------------------------------------------------------------------------
 // Time-varying retention: one step is  P <- g (a P) + x  with a real per-step factor g per
 // channel on top of the fixed rotation a; a segment is summarised by its end state and the

@@ -601,7 +601,8 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
         const float tau = prm.gate_tau;
         const bool want_mask = MASKED && prm.mask != nullptr;
         uint32_t *const mrow0 = prm.mask + ((long long)b * L + s0) * prm.MW + g * 2;
-        unsigned mkeep = 0u;                              // lane r: word 0 of row r; lane 16 + r: word 1
+        static_assert(T <= 16, "one 32-bit word per lane holds the gate bits of its rows");
+        unsigned mkeep = 0u;                              // bit pair i: this lane's gate bits of row i
         const bool second_word = g * 2 + 1 < prm.MW;
         const bool tap0 = Kc >= 4, tap1 = Kc >= 3, tap2 = Kc >= 2;
         // DYN: the rows' retention logits, all requested up front so that their latencies overlap
@@ -667,19 +668,7 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
                     float4 z;
                     const bool oA = push(plain, uA, vA, z.x, z.y), oB = push(plain, uB, vB, z.z, z.w);
                     xs[i * 32] = z;
-                    if (want_mask) {
-                        const unsigned bits = ((oA ? 1u : 0u) | (oB ? 2u : 0u)) << (2 * (lane & 15));
-                        const unsigned w0 = __reduce_or_sync(0xffffffffu, lane < 16 ? bits : 0u);
-                        const unsigned w1 = __reduce_or_sync(0xffffffffu, lane < 16 ? 0u : bits);
-                        // rows are parked in lanes and stored sixteen at a time
-                        if (lane == (i & 15)) mkeep = w0;
-                        if (lane == 16 + (i & 15)) mkeep = w1;
-                        if ((i & 15) == 15 || i == T - 1) {
-                            const int r = i - (i & 15) + (lane & 15);
-                            if ((lane & 15) <= (i & 15) && (FULL || r < nvalid) && (lane < 16 || second_word))
-                                mrow0[(long long)r * prm.MW + (lane >> 4)] = mkeep;
-                        }
-                    }
+                    mkeep |= ((oA ? 1u : 0u) | (oB ? 2u : 0u)) << (2 * i);     // this lane's gate bits of row i
                     if (FULL || i < nvalid) {
                         if constexpr (DYN) {
                             // e <- gamma_t (a e) + z, the factor pair kept for phase 3
@@ -696,6 +685,12 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
             }
         };
         if (Kc == 4 && !act) groups(std::true_type{}); else groups(std::false_type{});
+        if (want_mask) {
+            // the rows' mask words: lane r gets word 0 of row r, lane 16 + r word 1
+            const unsigned word = transpose_pairs16(mkeep, lane);
+            const int r = lane & 15;
+            if (r < T && (FULL || r < nvalid) && (lane < 16 || second_word)) mrow0[(long long)r * prm.MW + (lane >> 4)] = word;
+        }
     } else if constexpr (KIND == KIND_FWD) {
         // |p| >= eps decided as re^2 + im^2 >= eps^2 in double: both squares are exact there
         // and the sum rounds once, so the decision is reproducible bit for bit.  The fp32 sum
@@ -724,7 +719,8 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
         auto pass = [&](auto exact_tag, auto mask_tag) -> float {
             constexpr bool EXACT = decltype(exact_tag)::value, MASK = decltype(mask_tag)::value;
             float nearest = INFINITY;
-            unsigned mkeep = 0u;                          // lane r: word 0 of row r; lane 16 + r: word 1
+            static_assert(T <= 16, "one 32-bit word per lane holds the gate bits of its rows");
+            unsigned mkeep = 0u;                          // bit pair i: this lane's gate bits of row i
             e = zero4();
             dprod = make_float2(1.f, 1.f);
 #pragma unroll
@@ -757,20 +753,7 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
                 v.x = oA ? v.x : 0.f; v.y = oA ? v.y : 0.f;
                 v.z = oB ? v.z : 0.f; v.w = oB ? v.w : 0.f;
                 xs[i * 32] = v;                           // phase 3 reads the gated value
-                if (MASK) {
-                    // lanes 0..15 hold channels 0..31 of the group (word 0), lanes 16..31 word 1
-                    const unsigned bits = ((oA ? 1u : 0u) | (oB ? 2u : 0u)) << (2 * (lane & 15));
-                    const unsigned w0 = __reduce_or_sync(0xffffffffu, lane < 16 ? bits : 0u);
-                    const unsigned w1 = __reduce_or_sync(0xffffffffu, lane < 16 ? 0u : bits);
-                    // rows are parked in lanes and stored sixteen at a time
-                    if (lane == (i & 15)) mkeep = w0;
-                    if (lane == 16 + (i & 15)) mkeep = w1;
-                    if ((i & 15) == 15 || i == T - 1) {
-                        const int r = i - (i & 15) + (lane & 15);
-                        if ((lane & 15) <= (i & 15) && (FULL || r < nvalid) && (lane < 16 || second_word))
-                            mrow0[(long long)r * prm.MW + (lane >> 4)] = mkeep;
-                    }
-                }
+                if (MASK) mkeep |= ((oA ? 1u : 0u) | (oB ? 2u : 0u)) << (2 * i);   // this lane's gate bits of row i
                 if (FULL || i < nvalid) {
                     if constexpr (DYN) {
                         const float2 gm = make_float2(vA ? sigmoidf_fast(lg[i].x + fbA) : 0.f,
@@ -782,6 +765,13 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
                         e = cfma2(a, e, v);
                     }
                 }
+            }
+            if (MASK) {
+                // the rows' mask words (lanes 0..15 hold channels 0..31 of the group, word 0; lanes
+                // 16..31 word 1): lane r gets word 0 of row r, lane 16 + r word 1
+                const unsigned word = transpose_pairs16(mkeep, lane);
+                const int r = lane & 15;
+                if (r < T && (FULL || r < nvalid) && (lane < 16 || second_word)) mrow0[(long long)r * prm.MW + (lane >> 4)] = word;
             }
             return nearest;
         };
