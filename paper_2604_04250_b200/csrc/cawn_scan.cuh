@@ -328,6 +328,17 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
     static_assert(!LATE || (KIND == KIND_FWD && !DYN && !MASKED), "the late wait is built for the plain forward");
     const bool late_wait = LATE && early;
     if (!early) grid_wait_previous();
+    // Reverse kinds (they have waited already): the thread that later builds channel tid's
+    // coefficients asks for its gamma and theta now, and thread 0 for the epoch, so that the
+    // answers travel while the tile's copies are issued.
+    float pre_gamma = 1.f, pre_theta = 0.f;
+    if (REV && tid < 64 && g * 64 + tid < C) {
+        if (!DYN) pre_gamma = prm.gamma[g * 64 + tid];
+        pre_theta = prm.theta[g * 64 + tid];
+    }
+    unsigned long long epoch0 = 0;
+    unsigned hook0 = 0;
+    if (REV && tid == 0) ld_epoch_hook(prm.ws, epoch0, hook0);
     // Fused path: every warp stages its own T hidden rows (floats) behind kHalo rows of history in
     // the upper part of its own T x 512-byte slice of the tile, row r at byte 256 (T - 3) + 256 r
     // (r < kHalo: history).  The pushes the warp later writes into the same slice (row i at byte
@@ -470,9 +481,9 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
         const int ch = g * 64 + cl;
         double c1r = 0.0, c1i = 0.0, cTr = 0.0, cTi = 0.0, cAr = 0.0, cAi = 0.0;
         if (ch < C) {
-            const double gm = DYN ? 1.0 : (double)prm.gamma[ch];
+            const double gm = REV ? (double)pre_gamma : DYN ? 1.0 : (double)prm.gamma[ch];
             double sn, cs;
-            sincos((double)prm.theta[ch], &sn, &cs);
+            sincos(REV ? (double)pre_theta : (double)prm.theta[ch], &sn, &cs);
             c1r = gm * cs;
             c1i = REV ? -(gm * sn) : gm * sn;
             auto cpow = [](double br, double bi, int n, double &rr, double &ri) {
@@ -490,11 +501,9 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
     }
     // everything below touches what the previous launch may have written (workspace, states)
     if (early && KIND != KIND_FUSED && !late_wait) grid_wait_previous();
-    unsigned long long epoch0 = 0;
     unsigned arrived = 0;
     auto read_epoch = [&]() {                            // thread 0 only
-        unsigned hook0;
-        ld_epoch_hook(prm.ws, epoch0, hook0);
+        if (!REV) ld_epoch_hook(prm.ws, epoch0, hook0);
         sm.epoch = epoch0;
         sm.hook = hook0;
         // counted only once the epoch has been read (the increment depends on its value)
@@ -1170,6 +1179,20 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
             // three rows would need the tile after it in time, so their du (and the du of its three
             // earliest rows, for the tile before it) go to the edge area and the epilogue launch
             // finishes those rows.
+            // Every warp's partial sums go into its own rows of the saved-state tile, which only it
+            // read and which it has spent: 320 floats of conv sums, then the rotation sums, then the
+            // retention sums.  One barrier then serves the du rows and all the sums.
+            static_assert(T * 512 >= 2048, "a warp's spent rows hold its partial sums");
+            float *const part = reinterpret_cast<float *>(&sm.tile[1][w * T][0]);
+            constexpr int PSTRIDE = T * 128;             // floats between the warps' areas
+            if (prm.cpart != nullptr) {
+#pragma unroll
+                for (int j = 0; j < 5; ++j) { part[lane * 10 + j] = caA[j]; part[lane * 10 + 5 + j] = caB[j]; }
+            }
+            if (prm.qpart != nullptr) {
+                reinterpret_cast<float4 *>(part + 320)[lane] = qa;
+                if constexpr (DYN) reinterpret_cast<float2 *>(part + 448)[lane] = sacc_out;
+            }
             __syncthreads();
             const float4 (*du)[32] = sm.tile[0];
 #pragma unroll
@@ -1189,7 +1212,9 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
                     else { if (vA) __stcs(o, dA); if (vB) __stcs(o + 1, dB); }
                 }
             }
-            if (w == 0) {
+            // the sums over the warps, each in a fixed order, shared out among the warps
+            const float *const parts = reinterpret_cast<const float *>(&sm.tile[1][0][0]);
+            if (w == W - 1) {
                 const long long rem = L - (long long)k * TILE;
                 const int nrows = rem >= TILE ? TILE : (int)rem;           // rows this tile has
                 float *eg = prm.edge_du + (((long long)b * K + k) * 6) * C + c0;
@@ -1202,20 +1227,37 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
                 }
             }
             if (prm.cpart != nullptr) {
-                // per-tile sums for the conv gradients, in a fixed order (the P tile is spent)
-                __syncthreads();
-                float *sp = reinterpret_cast<float *>(&sm.tile[1][0][0]);
+                float *o = prm.cpart + (((long long)b * K + k) * C + c0) * 5;
+                for (int j = w; j < 10; j += W) {
+                    float acc = 0.f;
 #pragma unroll
-                for (int j = 0; j < 5; ++j) { sp[(w * 32 + lane) * 10 + j] = caA[j]; sp[(w * 32 + lane) * 10 + 5 + j] = caB[j]; }
-                __syncthreads();
-                if (w == 0) {
-                    float *o = prm.cpart + (((long long)b * K + k) * C + c0) * 5;
+                    for (int i = 0; i < W; ++i) acc += parts[i * PSTRIDE + lane * 10 + j];
+                    if (j < 5 ? vA : vB) o[j] = acc;
+                }
+            }
+            if (prm.qpart != nullptr) {
+                if (w == 2 % W) {
+                    float4 acc = reinterpret_cast<const float4 *>(parts + 320)[lane];
 #pragma unroll
-                    for (int j = 0; j < 10; ++j) {
-                        float acc = 0.f;
+                    for (int i = 1; i < W; ++i) {
+                        const float4 v = reinterpret_cast<const float4 *>(parts + i * PSTRIDE + 320)[lane];
+                        acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+                    }
+                    float2 *qp = prm.qpart + ((long long)b * K + k) * C + c0;
+                    if (vA) qp[0] = make_float2(acc.x, acc.y);
+                    if (vB) qp[1] = make_float2(acc.z, acc.w);
+                }
+                if constexpr (DYN) {
+                    if (prm.spart != nullptr && w == 3 % W) {
+                        float2 acc = reinterpret_cast<const float2 *>(parts + 448)[lane];
 #pragma unroll
-                        for (int i = 0; i < W; ++i) acc += sp[(i * 32 + lane) * 10 + j];
-                        if (j < 5 ? vA : vB) o[j] = acc;
+                        for (int i = 1; i < W; ++i) {
+                            const float2 v = reinterpret_cast<const float2 *>(parts + i * PSTRIDE + 448)[lane];
+                            acc.x += v.x; acc.y += v.y;
+                        }
+                        float *sp = prm.spart + ((long long)b * K + k) * C + c0;
+                        if (vA) sp[0] = acc.x;
+                        if (vB) sp[1] = acc.y;
                     }
                 }
             }
@@ -1252,7 +1294,7 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
             }
         }
     }
-    if constexpr (REV) {
+    if constexpr (REV && !MIX) {
         if (prm.qpart != nullptr) {
             __syncthreads();
             sm.sE[w][lane] = qa;
