@@ -355,50 +355,85 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
         const int Kh = prm.conv_k - 1;
         // a bf16 hidden value of a history row is kept as the float it widens to
         auto widen = [](unsigned short v) -> float { return __uint_as_float((unsigned)v << 16); };
-        // history rows that are earlier rows of h (they travel with the first group of own rows)
-#pragma unroll
-        for (int j = 0; j < kHalo; ++j) {
-            const long long t = s0 - kHalo + j;
-            float *d = hstage + j * 64;
-            if (j >= kHalo - Kh && t >= 0 && t < L) {
-                if constexpr (IN16) {
-                    const unsigned short *s16 = hin16 + ((long long)b * L + t) * C + c0;
-                    d[0] = vA ? widen(s16[0]) : 0.f;
-                    d[1] = vB ? widen(s16[1]) : 0.f;
-                } else {
-                    const float *src = hin + ((long long)b * L + t) * C + c0;
-                    if (vA) cp_async4(smem_addr(d), src); else d[0] = 0.f;
-                    if (vB) cp_async4(smem_addr(d + 1), src + 1); else d[1] = 0.f;
+        // float rows of whole 16-byte pieces: a half-warp copies one row's 256 bytes, a warp two
+        // rows per instruction (copies of 4 and 8 bytes take the slower path through L1); the lanes
+        // that read a row are then not the ones that brought it, so the warp synchronises after
+        // each wait
+        const bool wide = !IN16 && (C & 3) == 0 && (reinterpret_cast<uintptr_t>(prm.in) & 15) == 0;
+        if (wide) {
+            const int q4 = (lane & 15) * 4, hh = lane >> 4;
+            const bool cols = g * 64 + q4 < C;
+            float *const hbase = hstage - 2 * lane + q4;
+            auto history16 = [&](int j, bool on) {
+                const long long t = s0 - kHalo + j;
+                float *d = hbase + j * 64;
+                if (!on) return;
+                if (j >= kHalo - Kh && t >= 0 && t < L) {
+                    if (cols) cp_async16<0>(smem_addr(d), hin + ((long long)b * L + t) * C + g * 64 + q4);
+                    else *reinterpret_cast<float4 *>(d) = zero4();
+                } else if (t >= 0 || prm.tail_in == nullptr || j < kHalo - Kh) {
+                    *reinterpret_cast<float4 *>(d) = zero4();
                 }
-            } else if (t >= 0 || prm.tail_in == nullptr || j < kHalo - Kh) {
-                d[0] = 0.f; d[1] = 0.f;                 // no such tap, or no carried history
+            };
+            static_assert(kHalo == 3 && T % 2 == 0 && GR % 2 == 0, "rows go two to an instruction");
+            history16(hh, true);
+            history16(2, hh == 0);
+            const float *r = hin + ((long long)b * L + s0 + hh) * C + g * 64 + q4;
+#pragma unroll
+            for (int i = 0; i < T; i += 2) {
+                const bool row = FULL || i + hh < nvalid;
+                float *d = hbase + (kHalo + i + hh) * 64;
+                if (row && cols) cp_async16<0>(smem_addr(d), r); else *reinterpret_cast<float4 *>(d) = zero4();
+                r += 2 * (long long)C;
+                if ((i + 2) % GR == 0) cp_async_commit();
             }
         }
-        const float *r = hin + e0;
-        const unsigned short *r16 = hin16 + e0;
+        if (!wide) {
+            // history rows that are earlier rows of h (they travel with the first group of own rows)
 #pragma unroll
-        for (int i = 0; i < T; ++i) {
-            const bool row = FULL || i < nvalid;
-            float *d = hstage + (kHalo + i) * 64;
-            if constexpr (IN16) {
-                // the pair of bf16 goes into the first word of the slot; phase 1 widens it
-                if (VEC) {
-                    if (row && vA) cp_async4(smem_addr(d), r16); else d[0] = 0.f;
-                } else {
-                    unsigned lo = 0u, hi = 0u;
-                    if (row && vA) lo = r16[0];
-                    if (row && vB) hi = r16[1];
-                    reinterpret_cast<unsigned *>(d)[0] = lo | (hi << 16);
+            for (int j = 0; j < kHalo; ++j) {
+                const long long t = s0 - kHalo + j;
+                float *d = hstage + j * 64;
+                if (j >= kHalo - Kh && t >= 0 && t < L) {
+                    if constexpr (IN16) {
+                        const unsigned short *s16 = hin16 + ((long long)b * L + t) * C + c0;
+                        d[0] = vA ? widen(s16[0]) : 0.f;
+                        d[1] = vB ? widen(s16[1]) : 0.f;
+                    } else {
+                        const float *src = hin + ((long long)b * L + t) * C + c0;
+                        if (vA) cp_async4(smem_addr(d), src); else d[0] = 0.f;
+                        if (vB) cp_async4(smem_addr(d + 1), src + 1); else d[1] = 0.f;
+                    }
+                } else if (t >= 0 || prm.tail_in == nullptr || j < kHalo - Kh) {
+                    d[0] = 0.f; d[1] = 0.f;                 // no such tap, or no carried history
                 }
-                r16 += C;
-            } else if (VEC) {
-                if (row && vA) cp_async8<0>(smem_addr(d), r); else *reinterpret_cast<float2 *>(d) = make_float2(0.f, 0.f);
-            } else {
-                if (row && vA) cp_async4(smem_addr(d), r); else d[0] = 0.f;
-                if (row && vB) cp_async4(smem_addr(d + 1), r + 1); else d[1] = 0.f;
             }
-            r += C;
-            if ((i + 1) % GR == 0) cp_async_commit();
+            const float *r = hin + e0;
+            const unsigned short *r16 = hin16 + e0;
+#pragma unroll
+            for (int i = 0; i < T; ++i) {
+                const bool row = FULL || i < nvalid;
+                float *d = hstage + (kHalo + i) * 64;
+                if constexpr (IN16) {
+                    // the pair of bf16 goes into the first word of the slot; phase 1 widens it
+                    if (VEC) {
+                        if (row && vA) cp_async4(smem_addr(d), r16); else d[0] = 0.f;
+                    } else {
+                        unsigned lo = 0u, hi = 0u;
+                        if (row && vA) lo = r16[0];
+                        if (row && vB) hi = r16[1];
+                        reinterpret_cast<unsigned *>(d)[0] = lo | (hi << 16);
+                    }
+                    r16 += C;
+                } else if (VEC) {
+                    if (row && vA) cp_async8<0>(smem_addr(d), r); else *reinterpret_cast<float2 *>(d) = make_float2(0.f, 0.f);
+                } else {
+                    if (row && vA) cp_async4(smem_addr(d), r); else d[0] = 0.f;
+                    if (row && vB) cp_async4(smem_addr(d + 1), r + 1); else d[1] = 0.f;
+                }
+                r += C;
+                if ((i + 1) % GR == 0) cp_async_commit();
+            }
         }
         // history rows before t = 0 come from the carried tail: the previous call's output, never
         // read before that call is complete
@@ -444,11 +479,35 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
                 if (src != nullptr && vB) cp_async4(smem_addr(d + 1), src + 1); else d[1] = 0.f;
             }
         };
+        if ((C & 3) == 0 && ((reinterpret_cast<uintptr_t>(prm.hid) | reinterpret_cast<uintptr_t>(prm.tail_in)) & 15) == 0) {
+            // rows of whole 16-byte pieces: a half-warp copies one row's 256 bytes, a warp two rows
+            // per instruction (8-byte copies take the slower path through L1)
+            const int q4 = (lane & 15) * 4, hh = lane >> 4;
+            auto stage_h16 = [&](int R, bool on) {
+                const long long t = t_hi - R;
+                float *d = &sm.hrev[R][q4];
+                const float *src = nullptr;
+                if (t >= 0) src = prm.hid + ((long long)b * L + t) * C + g * 64 + q4;
+                else if (t >= -Kh && prm.tail_in != nullptr) src = prm.tail_in + ((long long)b * Kh + (Kh + t)) * C + g * 64 + q4;
+                if (on) {
+                    if (src != nullptr && g * 64 + q4 < C) cp_async16<0>(smem_addr(d), src);
+                    else *reinterpret_cast<float4 *>(d) = zero4();
+                }
+            };
+            static_assert(T % 2 == 0 && kHalo == 3, "rows go two to an instruction");
 #pragma unroll
-        for (int i = 0; i < T; ++i) stage_h(w * T + i);
-        if (w == 0) {
+            for (int i = 0; i < T; i += 2) stage_h16(w * T + i + hh, true);
+            if (w == W - 1) {
+                stage_h16(TILE + hh, true);
+                stage_h16(TILE + 2, hh == 0);
+            }
+        } else {
 #pragma unroll
-            for (int j = 0; j < kHalo; ++j) stage_h(TILE + j);
+            for (int i = 0; i < T; ++i) stage_h(w * T + i);
+            if (w == 0) {
+#pragma unroll
+                for (int j = 0; j < kHalo; ++j) stage_h(TILE + j);
+            }
         }
     }
     if constexpr (REV) {
@@ -605,6 +664,7 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
         const int Kc = prm.conv_k;
         // the first group of rows (and the history) has landed: the rolling window of the conv
         if (fused_tail_group) cp_async_wait_all(); else cp_async_wait_pending(NG - 1);
+        __syncwarp();                                     // rows may have been brought by other lanes
         float2 hv0 = hidden_row(0), hv1 = hidden_row(1), hv2 = hidden_row(2), hq[GR];
         const bool act = prm.clamp_silu != 0;
         const float tau = prm.gate_tau;
@@ -660,7 +720,7 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
             for (int gi = 0; gi < NG; ++gi) {
                 // the group's GR new hidden rows come out of the slice together, then the warp
                 // synchronises once: the pushes of these GR steps only reach rows read by now
-                if (gi > 0 && !fused_tail_group) cp_async_wait_pending(NG - 1 - gi);
+                if (gi > 0 && !fused_tail_group) { cp_async_wait_pending(NG - 1 - gi); __syncwarp(); }
 #pragma unroll
                 for (int q = 0; q < GR; ++q) hq[q] = hidden_row(gi * GR + kHalo + q);
                 __syncwarp();
