@@ -495,8 +495,19 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
                 }
             };
             static_assert(T % 2 == 0 && kHalo == 3, "rows go two to an instruction");
+            if (FULL) {
+                // every own row exists and is whole: one pointer, stepped two rows at a time
+                const float *src = prm.hid + ((long long)b * L + t_hi - (w * T + hh)) * C + g * 64 + q4;
+                const uint32_t d = smem_addr(&sm.hrev[w * T + hh][q4]);
 #pragma unroll
-            for (int i = 0; i < T; i += 2) stage_h16(w * T + i + hh, true);
+                for (int i = 0; i < T; i += 2) {
+                    cp_async16<0>(d + i * 256, src);
+                    src -= 2 * (long long)C;
+                }
+            } else {
+#pragma unroll
+                for (int i = 0; i < T; i += 2) stage_h16(w * T + i + hh, true);
+            }
             if (w == W - 1) {
                 stage_h16(TILE + hh, true);
                 stage_h16(TILE + 2, hh == 0);
@@ -513,8 +524,12 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
     if constexpr (REV) {
         float4 *const qs = &sm.tile[1][w * T][lane];
         const bool have = prm.aux != nullptr;
-        fetch_rows<VEC, T, 0>(qs, smem_addr(qs), reinterpret_cast<const char *>(prm.aux) + (e0 - C) * 8, rowbytes,
-                              vA, vB, [&](int i) { return have && (FULL || i < nvalid) && (t_first - i >= 1); });
+        if (FULL && have && t_first - (T - 1) >= 1)         // the common case: every row has a predecessor in the call
+            fetch_rows<VEC, T, 0>(qs, smem_addr(qs), reinterpret_cast<const char *>(prm.aux) + (e0 - C) * 8, rowbytes,
+                                  vA, vB, [](int) { return true; });
+        else
+            fetch_rows<VEC, T, 0>(qs, smem_addr(qs), reinterpret_cast<const char *>(prm.aux) + (e0 - C) * 8, rowbytes,
+                                  vA, vB, [&](int i) { return have && (FULL || i < nvalid) && (t_first - i >= 1); });
         cp_async_commit();
     }
 
