@@ -376,16 +376,30 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
                 }
             };
             static_assert(kHalo == 3 && T % 2 == 0 && GR % 2 == 0, "rows go two to an instruction");
-            history16(hh, true);
-            history16(2, hh == 0);
-            const float *r = hin + ((long long)b * L + s0 + hh) * C + g * 64 + q4;
+            if (FULL && Kh == kHalo && s0 >= kHalo) {
+                // a whole tile with all four taps behind kHalo earlier rows of the call: all T + kHalo
+                // rows exist and are whole, one pointer steps through them two rows at a time.  Copy
+                // group gi ends with the pair that holds the last row its steps read (row GR gi + GR + 2).
+                const float *src = hin + ((long long)b * L + s0 - kHalo + hh) * C + g * 64 + q4;
+                const uint32_t d = smem_addr(hbase + hh * 64);
 #pragma unroll
-            for (int i = 0; i < T; i += 2) {
-                const bool row = FULL || i + hh < nvalid;
-                float *d = hbase + (kHalo + i + hh) * 64;
-                if (row && cols) cp_async16<0>(smem_addr(d), r); else *reinterpret_cast<float4 *>(d) = zero4();
-                r += 2 * (long long)C;
-                if ((i + 2) % GR == 0) cp_async_commit();
+                for (int m = 0; m < (T + kHalo + 1) / 2; ++m) {
+                    if (2 * m + 1 < T + kHalo || hh == 0) cp_async16<0>(d + m * 512, src);
+                    src += 2 * (long long)C;
+                    if (m >= GR / 2 + 1 && (m - (GR / 2 + 1)) % (GR / 2) == 0) cp_async_commit();
+                }
+            } else {
+                history16(hh, true);
+                history16(2, hh == 0);
+                const float *r = hin + ((long long)b * L + s0 + hh) * C + g * 64 + q4;
+#pragma unroll
+                for (int i = 0; i < T; i += 2) {
+                    const bool row = FULL || i + hh < nvalid;
+                    float *d = hbase + (kHalo + i + hh) * 64;
+                    if (row && cols) cp_async16<0>(smem_addr(d), r); else *reinterpret_cast<float4 *>(d) = zero4();
+                    r += 2 * (long long)C;
+                    if ((i + 2) % GR == 0) cp_async_commit();
+                }
             }
         }
         if (!wide) {
