@@ -552,11 +552,19 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
     float wA[4] = {}, wB[4] = {}, bA = 0.f, bB = 0.f;
     if constexpr (KIND == KIND_FUSED) {
         const int Kc = prm.conv_k;
+        if (FULL && Kc == 4 && (reinterpret_cast<uintptr_t>(prm.conv_w) & 15) == 0) {
+            // four taps: the two channels' taps are two aligned 16-byte words
+            const float4 *w4 = reinterpret_cast<const float4 *>(prm.conv_w) + c0;
+            const float4 a4 = w4[0], b4 = w4[1];
+            wA[0] = a4.x; wA[1] = a4.y; wA[2] = a4.z; wA[3] = a4.w;
+            wB[0] = b4.x; wB[1] = b4.y; wB[2] = b4.z; wB[3] = b4.w;
+        } else {
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const int kk = j - (4 - Kc);
-            if (kk >= 0 && vA) wA[j] = prm.conv_w[(long long)c0 * Kc + kk];
-            if (kk >= 0 && vB) wB[j] = prm.conv_w[(long long)(c0 + 1) * Kc + kk];
+            for (int j = 0; j < 4; ++j) {
+                const int kk = j - (4 - Kc);
+                if (kk >= 0 && vA) wA[j] = prm.conv_w[(long long)c0 * Kc + kk];
+                if (kk >= 0 && vB) wB[j] = prm.conv_w[(long long)(c0 + 1) * Kc + kk];
+            }
         }
         if (prm.conv_bias != nullptr) { if (vA) bA = prm.conv_bias[c0]; if (vB) bB = prm.conv_bias[c0 + 1]; }
     }
@@ -922,11 +930,19 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
     float mwA[4] = {}, mwB[4] = {}, mbA = 0.f, mbB = 0.f;
     if constexpr (MIX) {
         const int Kc = prm.conv_k;
+        if (FULL && Kc == 4 && (reinterpret_cast<uintptr_t>(prm.conv_w) & 15) == 0) {
+            // four taps: the two channels' taps are two aligned 16-byte words
+            const float4 *w4 = reinterpret_cast<const float4 *>(prm.conv_w) + c0;
+            const float4 a4 = w4[0], b4 = w4[1];
+            mwA[0] = a4.x; mwA[1] = a4.y; mwA[2] = a4.z; mwA[3] = a4.w;
+            mwB[0] = b4.x; mwB[1] = b4.y; mwB[2] = b4.z; mwB[3] = b4.w;
+        } else {
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const int kk = j - (4 - Kc);
-            if (kk >= 0 && vA) mwA[j] = prm.conv_w[(long long)c0 * Kc + kk];
-            if (kk >= 0 && vB) mwB[j] = prm.conv_w[(long long)(c0 + 1) * Kc + kk];
+            for (int j = 0; j < 4; ++j) {
+                const int kk = j - (4 - Kc);
+                if (kk >= 0 && vA) mwA[j] = prm.conv_w[(long long)c0 * Kc + kk];
+                if (kk >= 0 && vB) mwB[j] = prm.conv_w[(long long)(c0 + 1) * Kc + kk];
+            }
         }
         if (prm.conv_bias != nullptr) { if (vA) mbA = prm.conv_bias[c0]; if (vB) mbB = prm.conv_bias[c0 + 1]; }
     }
