@@ -328,11 +328,13 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
     static_assert(!LATE || (KIND == KIND_FWD && !DYN && !MASKED), "the late wait is built for the plain forward");
     const bool late_wait = LATE && early;
     if (!early) grid_wait_previous();
-    // Reverse kinds (they have waited already): the thread that later builds channel tid's
-    // coefficients asks for its gamma and theta now, and thread 0 for the epoch, so that the
-    // answers travel while the tile's copies are issued.
+    // Reverse kinds (they have waited already) and the fused forward: the thread that later builds
+    // channel tid's coefficients asks for its gamma and theta now, and thread 0 for the epoch (the
+    // fused forward: once it has waited, below), so that the answers travel while the tile's
+    // copies are issued and land.  (The plain forward is bound by memory, not by this chain.)
+    constexpr bool PRE = REV || KIND == KIND_FUSED;
     float pre_gamma = 1.f, pre_theta = 0.f;
-    if (REV && tid < 64 && g * 64 + tid < C) {
+    if (PRE && tid < 64 && g * 64 + tid < C) {
         if (!DYN) pre_gamma = prm.gamma[g * 64 + tid];
         pre_theta = prm.theta[g * 64 + tid];
     }
@@ -452,6 +454,7 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
         // history rows before t = 0 come from the carried tail: the previous call's output, never
         // read before that call is complete
         if (early) grid_wait_previous();
+        if (tid == 0) ld_epoch_hook(prm.ws, epoch0, hook0);
         if (s0 < kHalo && prm.tail_in != nullptr) {
 #pragma unroll
             for (int j = 0; j < kHalo; ++j) {
@@ -577,9 +580,9 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
         const int ch = g * 64 + cl;
         double c1r = 0.0, c1i = 0.0, cTr = 0.0, cTi = 0.0, cAr = 0.0, cAi = 0.0;
         if (ch < C) {
-            const double gm = REV ? (double)pre_gamma : DYN ? 1.0 : (double)prm.gamma[ch];
+            const double gm = PRE ? (double)pre_gamma : DYN ? 1.0 : (double)prm.gamma[ch];
             double sn, cs;
-            sincos(REV ? (double)pre_theta : (double)prm.theta[ch], &sn, &cs);
+            sincos(PRE ? (double)pre_theta : (double)prm.theta[ch], &sn, &cs);
             c1r = gm * cs;
             c1i = REV ? -(gm * sn) : gm * sn;
             auto cpow = [](double br, double bi, int n, double &rr, double &ri) {
@@ -599,7 +602,7 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
     if (early && KIND != KIND_FUSED && !late_wait) grid_wait_previous();
     unsigned arrived = 0;
     auto read_epoch = [&]() {                            // thread 0 only
-        if (!REV) ld_epoch_hook(prm.ws, epoch0, hook0);
+        if (!PRE) ld_epoch_hook(prm.ws, epoch0, hook0);
         sm.epoch = epoch0;
         sm.hook = hook0;
         // counted only once the epoch has been read (the increment depends on its value)
