@@ -640,6 +640,32 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
         }
         return gm;
     };
+    // Where every 64-channel group lies inside one head (F a multiple of 64) the T logits a warp
+    // needs are one load: lane j fetches the logit of the warp's row j (lane T, for the reverse
+    // kinds, that of the row processed just before the first), and shuffles hand them round.
+    // (measured: a gain in the fused forward and the plain backward, a loss in the other two kinds)
+    const bool onehead = DYN && (KIND == KIND_FUSED || KIND == KIND_BWD) && (prm.F & 63) == 0;
+    float mylogit = 0.f;
+    if constexpr (DYN) {
+        if (onehead) {
+            long long t = REV ? t_first - lane : s0 + lane;
+            bool have = lane < T && (FULL || lane < nvalid);
+            if (REV && lane == T) { t = t_first + 1; have = t < L; }
+            if (have) mylogit = prm.gamma_logit[((long long)b * L + t) * prm.H + hA];
+        }
+    }
+    // the logits of this lane's two channels at the warp's row i (physical row t); 0 where there is no such row
+    auto row_logits = [&](int i, long long t) -> float2 {
+        float2 lg = make_float2(0.f, 0.f);
+        if (onehead) {
+            lg.x = lg.y = __shfl_sync(0xffffffffu, mylogit, i);
+        } else if (FULL || i < nvalid) {
+            const float *gl = prm.gamma_logit + ((long long)b * L + t) * prm.H;
+            if (vA) lg.x = gl[hA];
+            if (vB) lg.y = gl[hB];
+        }
+        return lg;
+    };
     float2 dprod = make_float2(1.f, 1.f);                // product of this thread's step factors
     float2 gfirst = make_float2(0.f, 0.f);               // DYN backward: factor of the row before this thread's first
 
@@ -718,14 +744,7 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
         float2 lgf[DYN ? T : 1];
         if constexpr (DYN) {
 #pragma unroll
-            for (int i = 0; i < T; ++i) {
-                lgf[i] = make_float2(0.f, 0.f);
-                if (FULL || i < nvalid) {
-                    const float *gl = prm.gamma_logit + ((long long)b * L + s0 + i) * prm.H;
-                    if (vA) lgf[i].x = gl[hA];
-                    if (vB) lgf[i].y = gl[hB];
-                }
-            }
+            for (int i = 0; i < T; ++i) lgf[i] = row_logits(i, s0 + i);
         }
         // One channel's push from its conv output u.  With q = e^-x: m = 1/(1+q) and
         // tanh x = 2/(1+q^2) - 1, so the phase is 2 pi r - pi with r = 1/(1+q^2), and
@@ -905,14 +924,25 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
             float2 lgb[T];
 #pragma unroll
             for (int i = 0; i < T; ++i) {
-                lgb[i] = make_float2(0.f, 0.f);
-                if (FULL || i < nvalid) {
-                    const float *gl = prm.gamma_logit + ((long long)b * L + (t_first - i)) * prm.H;
-                    if (vA) lgb[i].x = gl[hA];
-                    if (vB) lgb[i].y = gl[hB];
+                if constexpr (KIND == KIND_BWD) {
+                    lgb[i] = row_logits(i, t_first - i);
+                } else {
+                    lgb[i] = make_float2(0.f, 0.f);
+                    if (FULL || i < nvalid) {
+                        const float *gl = prm.gamma_logit + ((long long)b * L + (t_first - i)) * prm.H;
+                        if (vA) lgb[i].x = gl[hA];
+                        if (vB) lgb[i].y = gl[hB];
+                    }
                 }
             }
-            float2 gm = row_gamma(t_first + 1);
+            float2 gm;
+            if (KIND == KIND_BWD && onehead) {
+                const float lgp = __shfl_sync(0xffffffffu, mylogit, T);
+                const bool in = t_first + 1 < L;
+                gm = make_float2(in && vA ? sigmoidf_fast(lgp + fbA) : 0.f, in && vB ? sigmoidf_fast(lgp + fbB) : 0.f);
+            } else {
+                gm = row_gamma(t_first + 1);
+            }
             gfirst = gm;
 #pragma unroll
             for (int i = 0; i < T; ++i) {
