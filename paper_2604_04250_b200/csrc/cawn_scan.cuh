@@ -350,6 +350,7 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
     // No other warp touches the slice, so a warp starts as soon as its own first rows have landed.
     static_assert(KIND != KIND_FUSED || T == 16 || T == 4, "slice layout of the fused path is checked for 16 and 4 rows");
     float *const hstage = reinterpret_cast<float *>(&sm.tile[0][w * T][0]) + (T * 128 - (T + kHalo) * 64) + 2 * lane;
+    bool packed16 = false;                              // bf16 hidden rows of this warp sit packed, history included
     bool fused_tail_group = false;                      // this thread committed one more group (carried history)
     if constexpr (KIND == KIND_FUSED) {
         const float *hin = reinterpret_cast<const float *>(prm.in);
@@ -362,7 +363,23 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
         // that read a row are then not the ones that brought it, so the warp synchronises after
         // each wait
         const bool wide = !IN16 && (C & 3) == 0 && (reinterpret_cast<uintptr_t>(prm.in) & 15) == 0;
-        if (wide) {
+        // bf16 rows of a whole tile with all four taps behind kHalo earlier rows of the call: a row is
+        // 128 bytes, eight lanes copy it in 16-byte pieces, a warp four rows per instruction; every
+        // row, history included, then sits packed in the first half of its 256-byte slot.  Copy group
+        // gi ends with the instruction that holds the last row its steps read (row GR gi + GR + 2).
+        packed16 = IN16 && FULL && Kh == kHalo && s0 >= kHalo && (C & 7) == 0 && (reinterpret_cast<uintptr_t>(prm.in) & 15) == 0;
+        if (packed16) {
+            static_assert(GR == 4 && kHalo == 3, "four rows to an instruction, one instruction to a copy group");
+            const int p8 = (lane & 7) * 8, rr = lane >> 3;
+            const unsigned short *src = hin16 + ((long long)b * L + s0 - kHalo + rr) * C + g * 64 + p8;
+            const uint32_t d = smem_addr(hstage - 2 * lane + rr * 64 + (lane & 7) * 4);
+#pragma unroll
+            for (int m = 0; m < (T + kHalo + 3) / 4; ++m) {
+                if (4 * m + rr < T + kHalo) cp_async16<0>(d + m * 1024, src);
+                src += 4 * (long long)C;
+                if (m >= 1) cp_async_commit();
+            }
+        } else if (wide) {
             const int q4 = (lane & 15) * 4, hh = lane >> 4;
             const bool cols = g * 64 + q4 < C;
             float *const hbase = hstage - 2 * lane + q4;
@@ -404,7 +421,7 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
                 }
             }
         }
-        if (!wide) {
+        if (!wide && !packed16) {
             // history rows that are earlier rows of h (they travel with the first group of own rows)
 #pragma unroll
             for (int j = 0; j < kHalo; ++j) {
@@ -720,6 +737,7 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
         // input are still packed pairs)
         auto hidden_row = [&](int r) -> float2 {
             const float *slot = hstage + r * 64;
+            if (IN16 && packed16) return bf16x2_to_float2(reinterpret_cast<const unsigned *>(slot - 2 * lane)[lane]);
             if (IN16 && r >= kHalo) return bf16x2_to_float2(*reinterpret_cast<const unsigned *>(slot));
             return *reinterpret_cast<const float2 *>(slot);
         };
