@@ -45,6 +45,31 @@ def test_fused_shapes(B, L, C, Kc):
     check_fused(d, 0.1, P_in=P_in)
 
 
+def taps_at_8_byte_offset(monkeypatch):
+    """Make gpu_util.dev place every [C, 4] float array 8 bytes past a 16-byte boundary: the library
+    asks 8-byte alignment of the taps, and its 16-byte tap loads have to stand aside then."""
+    import torch
+    import gpu_util
+    real = gpu_util.dev
+
+    def dev8(a):
+        t = real(a)
+        if t is not None and t.ndim == 2 and t.shape[1] == 4 and t.dtype == torch.float32:
+            big = torch.empty(t.numel() + 2, dtype=t.dtype, device=t.device)
+            v = big[2:].view(t.shape)
+            v.copy_(t)
+            assert v.data_ptr() % 16 == 8
+            return v
+        return t
+    monkeypatch.setattr(gpu_util, "dev", dev8)
+
+
+def test_fused_taps_only_8_byte_aligned(monkeypatch):
+    taps_at_8_byte_offset(monkeypatch)
+    d = inputs.fused_inputs(2, 300, 192, seed=77, conv_k=4, with_tail=True, with_bias=True)
+    check_fused(d, 0.1)
+
+
 def test_fused_gate_closes_some_and_zero_state():
     d = inputs.fused_inputs(2, 2048, 128, seed=41)
     _, m_ref = check_fused(d, 0.1)

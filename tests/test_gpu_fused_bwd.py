@@ -95,6 +95,14 @@ def test_mixing_bwd_shapes(B, L, C, Kc):
     compare(got, reference(d, 0.1, P_in=d["P_in"], gso_P=d["gso_P"], gso_tail=tail), L, Kc)
 
 
+def test_mixing_bwd_taps_only_8_byte_aligned(monkeypatch):
+    from test_gpu_fused import taps_at_8_byte_offset
+    taps_at_8_byte_offset(monkeypatch)
+    d = make(2, 300, 192, 4, seed=1492)
+    got = run_mixing_bwd(d, 0.1, P_in=d["P_in"], gso_P=d["gso_P"], gso_tail=d["gso_tail"])
+    compare(got, reference(d, 0.1, P_in=d["P_in"], gso_P=d["gso_P"], gso_tail=d["gso_tail"]), 300, 4)
+
+
 @pytest.mark.parametrize("L", [15, 16, 17, 18, 19, 31, 32, 33, 34, 35, 63, 64, 65, 66, 67, 127, 128, 129, 130, 131, 192, 193])
 def test_mixing_bwd_rows_at_tile_seams(L):
     """Lengths around multiples of the tile (16 rows up to L = 32, 64 beyond): the rows whose conv
