@@ -287,8 +287,9 @@ def cfg2_prefill(cb, inputs, want, seconds):
     ncalls = 64
 
     def prefill(i):
+        st = torch.cuda.current_stream().cuda_stream      # looked up once per 64 calls, not per call
         for j in range(ncalls):
-            cb.cawn_phase_accumulate_fwd(prm, chunks[j % 16], g, t, ys[j % 4], ws, state_in=state, state_out=state)
+            cb.cawn_phase_accumulate_fwd(prm, chunks[j % 16], g, t, ys[j % 4], ws, state_in=state, state_out=state, stream=st)
     if want("cfg2"):
         tm, win = timed_blocks(prefill, 1, seconds, warmup=2)
         assert cb.cawn_poll_status(ws) == 0

@@ -34,6 +34,24 @@ cudaError_t launch_scan_inst(const ScanParams &sp, cudaStream_t st)
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
+    if constexpr (KIND == KIND_FUSED) {
+        // how many of these CTAs the device holds at once (asked once per device)
+        static int slots[64] = {};
+        ScanParams spf = sp;
+        if (dev >= 0 && dev < 64) {
+            if (slots[dev] == 0) {
+                int per_sm = 0, sms = 0;
+                if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, cawn_scan_kernel<T, W, KIND, VEC, MINB, DYN, EAR, IO, MASKED, LATE>,
+                                                                  W * 32, smem) == cudaSuccess &&
+                    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && per_sm > 0 && sms > 0)
+                    slots[dev] = per_sm * sms;
+                else
+                    slots[dev] = -1;
+            }
+            spf.first_wave = slots[dev] > 0 ? slots[dev] : 0;
+        }
+        return cudaLaunchKernelEx(&cfg, cawn_scan_kernel<T, W, KIND, VEC, MINB, DYN, EAR, IO, MASKED, LATE>, spf);
+    }
     return cudaLaunchKernelEx(&cfg, cawn_scan_kernel<T, W, KIND, VEC, MINB, DYN, EAR, IO, MASKED, LATE>, sp);
 }
 template <int T, int W, int KIND, int MINB, bool DYN = false, bool EAR = false, int IO = IO_F32, bool MASKED = true, bool LATE = false>

@@ -109,6 +109,7 @@ struct ScanParams {
     const float *freq_bias;      // [F]
     int H, F;
     float *grad_logit;           // BWD: [B][L][H]
+    int first_wave;              // fused forward: CTAs the device holds at once (0: unknown), set at launch
     int logit_direct;            // every 64-channel group holds whole heads: the logit gradient of a (row, head)
                                  // is complete in one warp and is stored; otherwise it is added atomically
                                  // into an array zeroed before the launch
@@ -327,7 +328,12 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
     // runs before the wait for the previous launch.
     static_assert(!LATE || (KIND == KIND_FWD && !DYN && !MASKED), "the late wait is built for the plain forward");
     const bool late_wait = LATE && early;
-    if (!early) grid_wait_previous();
+    // Fused forward: a CTA beyond the first wave starts in a slot that a CTA of this launch has
+    // left, and that one had waited for the previous launch: its own wait returns at once, so it
+    // waits (and asks for the epoch) before its copies instead of after them.
+    const bool wait_first = KIND == KIND_FUSED && early && prm.first_wave > 0 &&
+        (blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x >= (unsigned)prm.first_wave;
+    if (!early || wait_first) grid_wait_previous();
     // Reverse kinds (they have waited already) and the fused forward: the thread that later builds
     // channel tid's coefficients asks for its gamma and theta now, and thread 0 for the epoch (the
     // fused forward: once it has waited, below), so that the answers travel while the tile's
@@ -340,7 +346,7 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
     }
     unsigned long long epoch0 = 0;
     unsigned hook0 = 0;
-    if (REV && tid == 0) ld_epoch_hook(prm.ws, epoch0, hook0);
+    if ((REV || wait_first) && tid == 0) ld_epoch_hook(prm.ws, epoch0, hook0);
     // Fused path: every warp stages its own T hidden rows (floats) behind kHalo rows of history in
     // the upper part of its own T x 512-byte slice of the tile, row r at byte 256 (T - 3) + 256 r
     // (r < kHalo: history).  The pushes the warp later writes into the same slice (row i at byte
@@ -470,8 +476,8 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
         }
         // history rows before t = 0 come from the carried tail: the previous call's output, never
         // read before that call is complete
-        if (early) grid_wait_previous();
-        if (tid == 0) ld_epoch_hook(prm.ws, epoch0, hook0);
+        if (early && !wait_first) grid_wait_previous();
+        if (!wait_first && tid == 0) ld_epoch_hook(prm.ws, epoch0, hook0);
         if (s0 < kHalo && prm.tail_in != nullptr) {
 #pragma unroll
             for (int j = 0; j < kHalo; ++j) {
