@@ -356,6 +356,7 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
     // No other warp touches the slice, so a warp starts as soon as its own first rows have landed.
     static_assert(KIND != KIND_FUSED || T == 16 || T == 4, "slice layout of the fused path is checked for 16 and 4 rows");
     float *const hstage = reinterpret_cast<float *>(&sm.tile[0][w * T][0]) + (T * 128 - (T + kHalo) * 64) + 2 * lane;
+    bool in_packed = false;                             // bf16 pushes of this warp sit packed in the upper half of its slice
     bool packed16 = false;                              // bf16 hidden rows of this warp sit packed, history included
     bool fused_tail_group = false;                      // this thread committed one more group (carried history)
     if constexpr (KIND == KIND_FUSED) {
@@ -493,10 +494,29 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
             fused_tail_group = true;
         }
     } else {
-        if constexpr (IN16)
-            fetch_rows<VEC, T, GR, 0, true>(xs, smem_addr(xs), reinterpret_cast<const char *>(prm.in) + e0 * 4, rowbytes / 2,
-                                            vA, vB, [&](int i) { return FULL || i < nvalid; });
-        else
+        if constexpr (IN16) {
+            // Whole tiles of bf16 pushes whose rows are whole 16-byte pieces: a row is 256 bytes, a
+            // half-warp copies it, a warp two rows per instruction.  The T packed rows fill the upper
+            // half of the warp's T x 512-byte slice (row i at byte 256 T + 256 i); the gate pass widens
+            // row i into its 512-byte slot at byte 512 i, which only reaches packed rows 2i - T and
+            // 2i - T + 1 <= i: rows every lane has read by then (the warp synchronises after each read).
+            in_packed = FULL && (C & 3) == 0 && (reinterpret_cast<uintptr_t>(prm.in) & 15) == 0;
+            if (in_packed) {
+                static_assert(T % 2 == 0 && GR % 2 == 0, "rows go two to an instruction");
+                const int hh = lane >> 4;
+                const char *src = reinterpret_cast<const char *>(prm.in) + (((long long)b * L + s0 + hh) * C + g * 64) * 4 + (lane & 15) * 16;
+                const uint32_t d = smem_addr(&sm.tile[0][w * T][0]) + T * 256 + hh * 256 + (lane & 15) * 16;
+#pragma unroll
+                for (int m = 0; m < T / 2; ++m) {
+                    cp_async16<0>(d + m * 512, src);
+                    src += 8 * (long long)C;
+                    if ((2 * m + 2) % GR == 0) cp_async_commit();
+                }
+            } else {
+                fetch_rows<VEC, T, GR, 0, true>(xs, smem_addr(xs), reinterpret_cast<const char *>(prm.in) + e0 * 4, rowbytes / 2,
+                                                vA, vB, [&](int i) { return FULL || i < nvalid; });
+            }
+        } else
             fetch_rows<VEC, T, GR>(xs, smem_addr(xs), reinterpret_cast<const char *>(prm.in) + e0 * 8, rowbytes, vA, vB,
                                    [&](int i) { return FULL || i < nvalid; });
     }
@@ -879,6 +899,7 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
             for (int i = 0; i < T; ++i) {
                 if (!EXACT && i % GR == 0) {
                     cp_async_wait_pending(NG - 1 - i / GR);       // rows i .. i+GR-1 have landed
+                    if (IN16 && in_packed) __syncwarp();          // (brought by other lanes)
                     if (i == 0 && early_ptr != nullptr && !late_wait) {
                         er0 = ld_record(early_ptr + 2 * lane);
                         er1 = ld_record(early_ptr + 2 * lane + 1);
@@ -886,7 +907,13 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
                 }
                 float4 v;
                 if (IN16 && !EXACT) {                     // first touch: widen the staged bf16 in place
-                    const uint2 u = *reinterpret_cast<const uint2 *>(&xs[i * 32]);
+                    uint2 u;
+                    if (in_packed) {
+                        u = *reinterpret_cast<const uint2 *>(reinterpret_cast<const char *>(&sm.tile[0][w * T][0]) + T * 256 + i * 256 + lane * 8);
+                        __syncwarp();                     // every lane has read row i before any lane widens over it
+                    } else {
+                        u = *reinterpret_cast<const uint2 *>(&xs[i * 32]);
+                    }
                     const float2 cA = bf16x2_to_float2(u.x), cB = bf16x2_to_float2(u.y);
                     v = make_float4(cA.x, cA.y, cB.x, cB.y);
                 } else {
