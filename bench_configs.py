@@ -403,6 +403,20 @@ def cfg4_fused(cb, inputs, want, seconds, batch=0):
         assert cb.cawn_poll_status(ws) == 0
         out.append(record("cfg4_fused_bf16_in+out" + tag, B * L, B * L * C * 6, 1, tm, n, win))
         del h16, y16
+        # the paper's own layer form: bf16 network around the fp32 scan, per-token retention, Ear conv
+        dd = inputs.dynamic_retention_inputs(B, L, cfg.H, cfg.F, 7)
+        gl, fb = _dev(dd["gamma_logit"]), _dev(dd["freq_bias"])
+        prm16d = cb.make_params(B, L, cfg.H, cfg.F, gate_eps=cfg.gate_eps, gate_tau=tau, conv_k=cfg.conv_k,
+                                flags=IND | cb.CAWN_FLAG_RETENTION_DYNAMIC | cb.CAWN_FLAG_INPUT_BF16 | cb.CAWN_FLAG_OUTPUT_BF16)
+        ew, eb = dev_normal((2 * cfg.H, 3), 5), dev_normal((2 * cfg.H,), 6)
+        h16 = [h.to(torch.bfloat16) for h in hs]
+        z16 = [torch.empty((B, L, 2, C), dtype=torch.bfloat16, device="cuda") for _ in range(NS)]
+        tm, win = timed_blocks(lambda i: cb.cawn_phase_accumulate_fwd_ear(prm16d, h16[i % NS], None, t, ew, 3, z16[i % NS], ws, ear_bias=eb,
+                                                                          conv_w=w, gamma_logit=gl, freq_bias=fb), n, seconds, prewarm=8)
+        assert cb.cawn_poll_status(ws) == 0
+        out.append(record("cfg4_fused_dynamic_retention+ear_conv_bf16_in+out" + tag, B * L, B * L * (C * 6 + cfg.H * 4), 1, tm, n, win,
+                          note="the paper's layer form: bf16 hidden states in, bf16 planar Z out, fp32 scan, per-token retention"))
+        del h16, z16
     if want("cfg4bwd") or want("cfg4bwddyn"):
         h, P = hs[0], ys[0]
         prm_b = cb.make_params(B, L, cfg.H, cfg.F, gate_eps=cfg.gate_eps, gate_tau=tau, conv_k=cfg.conv_k)
