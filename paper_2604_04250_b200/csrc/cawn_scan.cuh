@@ -18,7 +18,10 @@
 //   3. every warp folds the window into the tile's carry-in, folds the earlier warps' ends on
 //      top, re-runs its T steps as the plain recurrence from that state and stores them
 //
-// A thread only ever touches the tile rows it copied itself, so the tile needs no barrier.
+// A warp only ever touches the tile rows it copied itself, so the tile needs no block barrier:
+// complex64 rows are copied and used by the same thread; hidden rows and bf16 rows are copied a
+// half-warp (or eight lanes) per row in 16-byte pieces, and the warp synchronises between waiting
+// for a copy group and using it.  (Copies of 4 or 8 bytes per lane issue far more slowly.)
 //
 // Carry window.  With M = kWindow, the tiles k = M, 2M, ... of a chain are checkpoints: they also
 // publish their carry-in X_k (the state before the tile).  Tile k reads the carry-in of the
@@ -523,7 +526,7 @@ __device__ __forceinline__ void scan_tile(const ScanParams &prm, ScanSmem<T, W, 
     if constexpr (MIX) {
         // hidden rows this tile's conv windows reach, in processing order: row R holds physical
         // row t_hi - R (t_hi = the tile's last row in time); before t = 0 comes the carried
-        // history, before that zeros.  Each thread brings its own T rows, warp 0 the kHalo more.
+        // history, before that zeros.  Each warp brings its own T rows, one warp the kHalo more.
         const int Kh = prm.conv_k - 1;
         const long long t_hi = L - 1 - (long long)k * TILE;
         auto stage_h = [&](int R) {
