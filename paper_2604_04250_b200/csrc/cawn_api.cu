@@ -138,7 +138,7 @@ cudaError_t launch_epilogue(EpilogueParams ep, bool want_q, bool want_s, bool wa
     ep.nb_s = want_s ? (ep.F + kEpiFW - 1) / kEpiFW : 0;
     ep.nb_c = want_c ? (ep.C + kEpiCW - 1) / kEpiCW : 0;
     ep.nb_ex = (ep.C + kEpiWarps * 32 - 1) / (kEpiWarps * 32);
-    const long long seams = want_seams ? (long long)ep.nb_ex * (ep.K + 1) * ep.B : 0;
+    const long long seams = want_seams ? (long long)ep.nb_ex * ((ep.K + kEpiSeams) / kEpiSeams) * ep.B : 0;
     const long long blocks = (long long)ep.nb_q + ep.nb_s + ep.nb_c + seams;
     if (blocks == 0) return cudaSuccess;
     if (blocks > 2147483647ll) return cudaErrorInvalidValue;

@@ -24,6 +24,7 @@ namespace cawn {
 constexpr int kEpiWarps = 32;
 constexpr int kEpiCW = 8;            // channels per block of the q and c jobs
 constexpr int kEpiFW = 2;            // harmonics per block of the s job
+constexpr int kEpiSeams = 4;         // seams per thread of the seam job: their loads are issued together
 struct EpilogueParams {
     int nb_q, nb_s, nb_c, nb_ex;     // blocks per job; nb_ex: blocks along the channels of one seam
     int nparts, C, H, F, Kc;
@@ -71,8 +72,10 @@ __device__ __forceinline__ void block_sum_fixed_order(double (&v)[NV], double *s
 //   call's last conv_k-1 rows)          for those rows (kb < K), and
 //   grad of the carried history rows s = -Kh .. -1 (kb = K), which collect from du(0..2)
 //   and, when the call is shorter than the history, pass part of the incoming gradient through.
-// One thread per channel; taps right-aligned as in the scan kernel.
-__device__ __forceinline__ void seam_rows(const EpilogueParams &ep, int c, int kb, int b)
+// One thread per channel and kEpiSeams adjacent seams (kb0 .. kb0 + kEpiSeams - 1, those <= K): the
+// du values of all of them are requested before the first is used.  Taps right-aligned as in the
+// scan kernel.
+__device__ __forceinline__ void seam_rows(const EpilogueParams &ep, int c, int kb0, int b)
 {
     const int C = ep.C, K = ep.K, tile = ep.tile, Kc = ep.Kc, Kh = Kc - 1;
     const long long L = ep.L;
@@ -100,36 +103,47 @@ __device__ __forceinline__ void seam_rows(const EpilogueParams &ep, int c, int k
         if (r - t_lo < 3) return e[(3 + (r - t_lo)) * C];
         return 0.f;                                  // not an edge row: never asked for
     };
-    if (kb < K) {
-        // The three latest rows of tile kb, t_hi - i (i = 0, 1, 2), reach du of rows t_hi + 3 .. t_hi - 2:
-        // the three earliest rows of the tile after it in time (tile kb - 1, its second edge triple)
-        // and this tile's own three latest (its first edge triple; rows it does not have hold 0).
+    // The three latest rows of tile kb, t_hi - i (i = 0, 1, 2), reach du of rows t_hi + 3 .. t_hi - 2:
+    // the three earliest rows of the tile after it in time (tile kb - 1, its second edge triple)
+    // and this tile's own three latest (its first edge triple; rows it does not have hold 0).
+    float d[kEpiSeams][6];                           // d[s][m + 2] = du(t_hi + m) of seam kb0 + s, m = -2 .. 3
+#pragma unroll
+    for (int s = 0; s < kEpiSeams; ++s) {
+        const int kb = kb0 + s;
+#pragma unroll
+        for (int i = 0; i < 6; ++i) d[s][i] = 0.f;
+        if (kb < K) {
+            const float *own = ep.edge_du + (((long long)b * K + kb) * 6) * C + c;
+#pragma unroll
+            for (int i = 0; i < 3; ++i) d[s][2 - i] = __ldg(own + (long long)i * C);
+            if (kb > 0) {
+                const float *nxt = own - 3ll * C;     // the second edge triple of tile kb - 1
+#pragma unroll
+                for (int i = 0; i < 3; ++i) d[s][3 + i] = __ldg(nxt + (long long)i * C);
+            }
+        }
+    }
+#pragma unroll
+    for (int s = 0; s < kEpiSeams; ++s) {
+        const int kb = kb0 + s;
+        if (kb >= K) continue;
         const long long t_hi = L - 1 - (long long)kb * tile;
         long long t_lo = L - (long long)(kb + 1) * tile;
         if (t_lo < 0) t_lo = 0;
-        const float *own = ep.edge_du + (((long long)b * K + kb) * 6) * C + c;
-        float d[6];                                  // d[m + 2] = du(t_hi + m), m = -2 .. 3
-#pragma unroll
-        for (int i = 0; i < 3; ++i) d[2 - i] = own[(long long)i * C];
-        if (kb > 0) {
-            const float *nxt = ep.edge_du + (((long long)b * K + (kb - 1)) * 6 + 3) * C + c;
-#pragma unroll
-            for (int i = 0; i < 3; ++i) d[3 + i] = nxt[(long long)i * C];
-        } else {
-            d[3] = d[4] = d[5] = 0.f;
-        }
 #pragma unroll
         for (int i = 0; i < 3; ++i) {
             const long long srow = t_hi - i;
             if (srow >= t_lo) {
                 float acc = 0.f;
 #pragma unroll
-                for (int j = 0; j < 4; ++j) acc = fmaf(wt[j], d[(3 - i - j) + 2], acc);
+                for (int j = 0; j < 4; ++j) acc = fmaf(wt[j], d[s][(3 - i - j) + 2], acc);
                 if (ep.dtail_out != nullptr && srow >= L - Kh) acc += ep.dtail_out[((long long)b * Kh + (srow - (L - Kh))) * C + c];
                 ep.grad_h[((long long)b * L + srow) * C + c] = acc;
             }
         }
-    } else if (ep.dtail_in != nullptr) {
+    }
+    if (kb0 + kEpiSeams <= K) return;                // seam K (the carried history) is not in this group
+    if (ep.dtail_in != nullptr) {
         for (int r = 0; r < Kh; ++r) {
             const long long s = r - Kh;
             float acc = 0.f;
@@ -217,10 +231,11 @@ __global__ void __launch_bounds__(kEpiWarps * 32) cawn_bwd_epilogue_kernel(const
     }
     blk -= ep.nb_c;
     {
+        const int groups = (ep.K + kEpiSeams) / kEpiSeams;       // seams 0 .. K in groups of kEpiSeams
         const int cb = blk % ep.nb_ex, rest = blk / ep.nb_ex;
-        const int kb = rest % (ep.K + 1), b = rest / (ep.K + 1);
+        const int kg = rest % groups, b = rest / groups;
         const int c = cb * (kEpiWarps * 32) + threadIdx.x;
-        if (c < C && b < ep.B) seam_rows(ep, c, kb, b);
+        if (c < C && b < ep.B) seam_rows(ep, c, kg * kEpiSeams, b);
     }
 }
 
